@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of BPT graph self-attention (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config NAME]
+
+One step = one forward and one backward pass of the whole hot path over one batch of
+seeded synthetic input.  The default workload is the character-level-LM-shaped layer
+(batch 4, n = 8192, k = 64, left-only, 8 heads x 64, bf16).  Prints ONE JSON line.
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank processes
+its own batch of the same shape (weak scaling); the only exchange is the all-reduce of
+the relation-embedding gradient, which is shared by the whole batch.
+
+`--impl reference` times the fp64 CPU oracle on the host cores on a bounded sample of
+the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "BPT graph-attention fwd+bwd edges/sec"
+UNIT = "edges/s"
+GATHER_BYTES_PER_EDGE_HEAD = {  # algorithmic bytes of the gather model, per edge and head
+    "fwd": lambda d, s: 2 * d * s,            # K row + V row
+    "bwd_dst": lambda d, s: 2 * d * s,        # K row + V row again
+    "bwd_src": lambda d, s: 2 * d * s + 8,    # Q row + dO row + (P, dS) or (lse, delta)
+}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def all_configs():
+    from paper_1911_04070_b200 import synth
+    c = dict(synth.CONFIGS)
+    c.update(synth.sweep_configs())
+    return c
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples during the timed region."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def run_reference(args, cfg_name, cfg):
+    """The fp64 oracle (plain C, OpenMP over batch x head) on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ctwin
+    from paper_1911_04070_b200 import synth
+    g = ctwin.CGraph(cfg["n"], cfg["k"], cfg["flags"])
+    Bs = 1  # bounded sample: one batch entry per step (entries are independent)
+    x = synth.make_inputs(Bs, g.n_nodes, cfg["H"], cfg["d"], g.n_rel, seed=cfg["seed"], std_qkv=cfg["std_qkv"], bf16=cfg["bf16"])
+    scale = cfg["d"] ** -0.5
+    x64 = {a: np.ascontiguousarray(b, dtype=np.float64) for a, b in x.items()}
+
+    def step():
+        ctwin.attn_fwd(g, x64["q"], x64["k"], x64["v"], x64["rel_emb"], scale)
+        if cfg["backward"]:
+            ctwin.attn_bwd(g, x64["q"], x64["k"], x64["v"], x64["rel_emb"], scale, x64["d_out"])
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = Bs * g.n_edges / dt
+    cores = ctwin.threads()
+    sample = "1 of %d batch entries per step (entries are independent), full n, all heads" % cfg["B"]
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg_name, "n": cfg["n"], "k": cfg["k"], "left_only": bool(cfg["flags"] & 1), "batch": Bs,
+                   "heads": cfg["H"], "d_head": cfg["d"], "pass": "fwd+bwd" if cfg["backward"] else "fwd"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cpu_baseline(cfg):
+    from oracle import ctwin
+    from paper_1911_04070_b200 import synth
+    g = ctwin.CGraph(cfg["n"], cfg["k"], cfg["flags"])
+    Bs = min(cfg["B"], 2)
+    x = synth.make_inputs(Bs, g.n_nodes, cfg["H"], cfg["d"], g.n_rel, seed=cfg["seed"], std_qkv=cfg["std_qkv"], bf16=cfg["bf16"])
+    x64 = {a: np.ascontiguousarray(b, dtype=np.float64) for a, b in x.items()}
+    scale = cfg["d"] ** -0.5
+    t0 = time.perf_counter()
+    ctwin.attn_fwd(g, x64["q"], x64["k"], x64["v"], x64["rel_emb"], scale)
+    if cfg["backward"]:
+        ctwin.attn_bwd(g, x64["q"], x64["k"], x64["v"], x64["rel_emb"], scale, x64["d_out"])
+    dt = time.perf_counter() - t0
+    return {"value": Bs * g.n_edges / dt, "unit": UNIT, "cores": ctwin.threads(), "kind": "oracle",
+            "sample": "%d of %d batch entries, one pass, %.1f s" % (Bs, cfg["B"], dt)}
+
+
+def run_ours(args, cfg_name, cfg):
+    import torch
+    import torch.distributed as dist
+    from paper_1911_04070_b200 import binding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    B, H, d = cfg["B"], cfg["H"], cfg["d"]
+    do_bwd = cfg["backward"]
+    g = binding.bpt_build_graph(cfg["n"], cfg["k"], cfg["flags"], device=dev, with_transpose=do_bwd)
+    E, N = g.n_edges, g.n_nodes
+    dt_t = torch.bfloat16 if cfg["bf16"] else torch.float32
+    esize = 2 if cfg["bf16"] else 4
+    x = synth.make_inputs(B, N, H, d, g.n_rel, seed=cfg["seed"] + 1000 * rank, std_qkv=cfg["std_qkv"], bf16=cfg["bf16"], with_grad=do_bwd)
+    host = {a: torch.from_numpy(b).to(dt_t).pin_memory() for a, b in x.items()}
+    del x
+    t = {a: b.to(dev, non_blocking=True) for a, b in host.items()}
+    scale = d ** -0.5
+    code = binding.BPT_BF16 if cfg["bf16"] else binding.BPT_F32
+    ws_f = binding.bpt_attn_workspace_bytes(g, B, H, d, code, False)
+    ws_b = binding.bpt_attn_workspace_bytes(g, B, H, d, code, True) if do_bwd else 0
+    ws = torch.empty(max(ws_f, ws_b, 1), dtype=torch.uint8, device=dev)
+    out = torch.empty_like(t["q"])
+    lse = torch.empty((B, N, H), dtype=torch.float32, device=dev)
+    dq, dk, dv = (torch.empty_like(t["q"]) for _ in range(3))
+    d_rel = torch.empty((g.n_rel, d), dtype=torch.float32, device=dev)
+
+    def step():
+        binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out=out, lse=lse, workspace=ws)
+        if do_bwd:
+            binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"], workspace=ws,
+                                 dq=dq, dk=dk, dv=dv, d_rel=d_rel)
+            if world > 1:
+                dist.all_reduce(d_rel)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        v = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(v, op=dist.ReduceOp.MAX)
+        return float(v.item())
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+
+    # ---- timed region: K steps, device-resident inputs ---------------------------------
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    cap = min(args.steps * 8 + 8, 4000)
+    binding.bpt_trace_begin(cap)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    marks = binding.bpt_trace_end(cap)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_step = ms_total / args.steps
+    value = world * B * E / (ms_step * 1e-3)
+
+    # ---- end to end: host buffers in, results back to the host, every step --------------
+    names_in = ["q", "k", "v", "rel_emb"] + (["d_out"] if do_bwd else [])
+    res_dev = [out, lse] + ([dq, dk, dv, d_rel] if do_bwd else [])
+    res_host = [torch.empty(r.shape, dtype=r.dtype).pin_memory() for r in res_dev]
+    h2d = sum(host[a].numel() * host[a].element_size() for a in names_in)
+    d2h = sum(r.numel() * r.element_size() for r in res_dev)
+
+    def e2e_step():
+        for a in names_in:
+            t[a].copy_(host[a], non_blocking=True)
+        step()
+        for rd, rh in zip(res_dev, res_host):
+            rh.copy_(rd, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-kernel shares and the roofline of the dominant kernel --------------------
+    per = {}
+    for name, ms in marks:
+        per.setdefault(name, []).append(ms)
+    kernels = {name: {"launches": len(v), "avg_ms": sum(v) / len(v), "share": sum(v) / max(sum(m for _, m in marks), 1e-9)}
+               for name, v in per.items()}
+    dominant = max(kernels, key=lambda a: kernels[a]["avg_ms"] * kernels[a]["launches"]) if kernels else None
+    peak, peak_kind = load_peaks()
+    roofline = None
+    if dominant:
+        key = "fwd" if dominant.startswith("fwd") else ("bwd_dst" if "dst" in dominant else "bwd_src")
+        alg_bytes = GATHER_BYTES_PER_EDGE_HEAD[key](d, esize) * B * H * E
+        achieved = alg_bytes / (kernels[dominant]["avg_ms"] * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
+                    "unit": "GB/s", "frac": achieved / peak, "traffic": None,
+                    "model": "gathered K/V (or Q/dO) rows per edge and head, no on-chip reuse credited"}
+    # whole-step fraction of the gather-model roofline (the target figure of the benchmark definition)
+    gathered = sum(GATHER_BYTES_PER_EDGE_HEAD[a](d, esize) for a in (["fwd", "bwd_dst", "bwd_src"] if do_bwd else ["fwd"])) * B * H * E
+    step_roof_ms = gathered / (peak * 1e9) * 1e3
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if cfg["bf16"] else "f32", "data": "synthetic",
+        "config": {"workload": cfg_name, "n": cfg["n"], "k": cfg["k"], "left_only": bool(cfg["flags"] & 1),
+                   "batch_per_gpu": B, "heads": H, "d_head": d, "edges_per_sequence": E,
+                   "pass": "fwd+bwd" if do_bwd else "fwd", "l2": "inputs larger than L2", "parallelism": "batch shards x%d" % world},
+        "edge_heads_per_s": value * H, "tokens_per_s": world * B * cfg["n"] / (ms_step * 1e-3),
+        "hbm_roofline_frac_step": step_roof_ms / ms_step, "hbm_roofline_ms_step": step_roof_ms,
+        "clocks": clocks,
+        "e2e": {"value": world * B * E / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": len(marks),
+        "kernels": kernels,
+        "roofline": roofline,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(cfg)
+    print(json.dumps(result))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="cfg4_char_lm")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    cfgs = all_configs()
+    if args.config not in cfgs:
+        raise SystemExit("unknown config %s; choose from %s" % (args.config, ", ".join(sorted(cfgs))))
+    cfg = cfgs[args.config]
+    if args.impl == "reference":
+        run_reference(args, args.config, cfg)
+    else:
+        if args.warmup < 3:
+            args.warmup = 3
+        run_ours(args, args.config, cfg)
+
+
+if __name__ == "__main__":
+    main()

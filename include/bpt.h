@@ -1,0 +1,159 @@
+/*
+ * bpt.h -- C ABI of the B200 (sm_100a) implementation of BP-Transformer's graph
+ * self-attention (arXiv 1911.04070).
+ *
+ * The library builds the binary-partition attention graph of Sec. 3.2 on the
+ * device and evaluates graph self-attention with tree relative positions
+ * (Sec. 3.1 and 3.4) forward and backward over it.
+ *
+ * Conventions (0-indexed): n tokens (a power of two), L = log2 n, node (l, m)
+ * is the m-th node of level l and covers tokens [m*2^l, (m+1)*2^l); level 0 are
+ * the tokens, level L is the root.  Node ids are level-major:
+ *     id(l, m) = 2n - (2n >> l) + m        (tokens 0..n-1, root 2n-2).
+ * An edge v -> u means "u attends to v".
+ *
+ * Ownership: the caller owns every buffer.  Unless a comment says "host", every
+ * pointer is a DEVICE pointer valid on the current device.  Calls enqueue work on
+ * `cuda_stream` (a cudaStream_t passed as void*, NULL = legacy default stream) and
+ * return without synchronising.  Nothing is allocated or kept between calls.
+ * Argument errors are detected on the host before anything is launched.
+ */
+#ifndef BPT_H
+#define BPT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BPT_OK = 0,
+    BPT_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, n not a power of two, ... */
+    BPT_ERR_UNSUPPORTED = 2,  /* head size / dtype / range the kernels do not cover        */
+    BPT_ERR_WORKSPACE = 3,    /* workspace missing or smaller than the size query says      */
+    BPT_ERR_CUDA = 4,         /* a CUDA runtime call or launch failed                       */
+    BPT_ERR_TIMEOUT = 5,      /* reserved: a bounded device-side wait expired               */
+    BPT_ERR_OVERFLOW = 6      /* edge count does not fit the 32-bit index arrays            */
+} bpt_status;
+
+/* flags of a graph */
+enum {
+    BPT_BIDIR = 0,      /* contextual edges from both sides (Sec. 3.2.2)                          */
+    BPT_LEFT_ONLY = 1,  /* only the left context, for autoregressive use (Sec. 4.2); self and      */
+                        /* affiliated edges are kept                                               */
+    BPT_MODE_PAD = 0,   /* default: k nodes per level plus the extra node that aligns the next     */
+                        /* level with a whole parent ("when the index p_l+k-1 is odd...", 3.2.2)   */
+    BPT_MODE_ALG1 = 2   /* Algorithm 1 taken literally: exactly k nodes per level, no extra node   */
+};
+
+typedef enum { BPT_F32 = 0, BPT_BF16 = 1 } bpt_dtype;
+
+typedef struct {
+    int32_t n, k;
+    uint32_t flags;
+    int32_t n_levels;             /* L = log2 n                                     */
+    int32_t n_nodes;              /* 2n - 1 (Sec. 3.2.1)                            */
+    int32_t n_rel;                /* rows of the relation table, see bpt_build_graph */
+    int64_t n_edges;              /* E                                              */
+    size_t build_workspace_bytes; /* workspace bpt_build_graph needs                */
+} bpt_graph_dims;
+
+typedef struct {
+    const int32_t* row_ptr; /* [n_nodes + 1] CSR by destination                              */
+    const int32_t* col;     /* [E] source node of each edge, ascending inside a row          */
+    const int32_t* rel;     /* [E] relation id of each edge                                  */
+    const int32_t* t_ptr;   /* [n_nodes + 1] by-source lists (needed by the backward), or NULL */
+    const int32_t* t_dst;   /* [E] destination node, ascending inside a source's list        */
+    const int32_t* t_eid;   /* [E] position of that edge in col/rel                          */
+    bpt_graph_dims dims;
+} bpt_graph;
+
+/*
+ * Sizes of the graph for (n, k, flags) -- host only, no device work.
+ * Sec. 3.2: 2n-1 nodes; per token a self loop (Algorithm 1, N <- {u}), k (or k+1
+ * with the pad rule) contextual nodes per level and side, fine to coarse; per span
+ * one affiliated edge from every token it contains.
+ * Requires n a power of two, 2 <= n <= 2^20, 1 <= k <= 2^20.  `out` is a host pointer.
+ * Errors: INVALID_ARG, UNSUPPORTED (range), OVERFLOW (E >= 2^31).
+ */
+bpt_status bpt_graph_dims_query(int32_t n, int32_t k, uint32_t flags, bpt_graph_dims* out);
+
+/*
+ * Build the graph on the device (Sec. 3.2.2 edge construction, Sec. 3.4 labels).
+ *
+ * Outputs (device, caller-allocated): row_ptr[n_nodes+1], col[E], rel[E] and, unless
+ * all three are NULL, the by-source lists t_ptr[n_nodes+1], t_dst[E], t_eid[E].
+ * Rows are destinations in node-id order, sources ascending by node id.
+ * Relation ids, with W = k+1:  self = 0;  o-th node (nearest first) joining on the
+ * left at level j: 1 + j*W + o;  on the right: 1 + L*W + j*W + o;  token -> its
+ * ancestor at level j (1..L): 1 + 2*L*W + (j-1);  n_rel = 1 + 2*L*W + L.
+ * `dims` (host) must come from bpt_graph_dims_query.  `workspace` (device) must hold
+ * dims->build_workspace_bytes.  `out` (host) receives the pointers and dims.
+ * Errors: INVALID_ARG, WORKSPACE, CUDA.
+ */
+bpt_status bpt_build_graph(const bpt_graph_dims* dims, int32_t* row_ptr, int32_t* col, int32_t* rel,
+                           int32_t* t_ptr, int32_t* t_dst, int32_t* t_eid,
+                           void* workspace, void* cuda_stream, bpt_graph* out);
+
+/*
+ * Bytes of device workspace bpt_attn_fwd (backward == 0) or bpt_attn_bwd
+ * (backward != 0) needs for this problem; 0 on invalid arguments.  Host only.
+ */
+size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype, int backward);
+
+/*
+ * Forward graph self-attention with relative positions (Sec. 3.4 equation, built on
+ * the GSA equations of Sec. 3.1).  For every batch entry b, node u, head h:
+ *     s_e = scale * q[b,u,h,:] . (k[b,v,h,:] + rel_emb[rel_e,:])   over edges e = (v -> u)
+ *     P   = softmax_e(s),   out[b,u,h,:] = sum_e P_e v[b,v,h,:],   lse[b,u,h] = log sum_e exp(s_e)
+ * q, k, v, out: [B, n_nodes, H, d] contiguous, element type `dtype`; rel_emb: [n_rel, d],
+ * same type, shared by all heads; lse: [B, n_nodes, H] fp32.  Accumulation is fp32.
+ * `scale` is explicit (the paper divides by sqrt(d); callers pass 1/sqrt(d)).
+ * d must be 32 or 64.  `g` is a host pointer to a struct of device pointers.
+ * `workspace` may be NULL when the size query returns 0.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ */
+bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                        const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                        void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward of the same equation: given d_out = dLoss/d out, with P_e = exp(s_e - lse_u),
+ *     dP_e = d_out_u . v_v,   dS_e = P_e (dP_e - d_out_u . out_u),
+ *     dq_u = scale * sum_{e into u} dS_e (k_v + rel_emb[rel_e]),
+ *     dk_v = scale * sum_{e out of v} dS_e q_u,      dv_v = sum_{e out of v} P_e d_out_u,
+ *     d_rel[r] = scale * sum_{b,h} sum_{e: rel_e = r} dS_e q_u     (the table is shared, Sec. 3.4).
+ * out and lse are the forward's results.  dq, dk, dv: [B, n_nodes, H, d] in `dtype`;
+ * d_rel: [n_rel, d] fp32.  All four are overwritten, not accumulated into.  The sums are
+ * taken in a fixed order without atomics, so results are bit-reproducible.
+ * The graph must carry the by-source lists.  Errors as for the forward.
+ */
+bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                        const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                        const void* out, const float* lse, const void* d_out,
+                        void* dq, void* dk, void* dv, float* d_rel,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Per-launch timing for benchmarks (no counterpart in the paper).  Between
+ * bpt_trace_begin and bpt_trace_end every kernel the library launches is followed by
+ * a CUDA event on its stream; bpt_trace_end waits for the last one and returns, for
+ * the first min(*n_marks, capacity) launches, the milliseconds since the previous
+ * mark (ms, host array, may be NULL) and a static name (names, host array, may be
+ * NULL).  `capacity` of bpt_trace_begin bounds the number of launches recorded
+ * (< 4096); later launches go unrecorded.  This is the one piece of process-global
+ * state in the library: not thread-safe, off by default, one trace at a time.
+ * Errors: INVALID_ARG (nesting, capacity), CUDA.
+ */
+bpt_status bpt_trace_begin(int32_t capacity, void* cuda_stream);
+bpt_status bpt_trace_end(int32_t* n_marks, float* ms, const char** names, int32_t capacity);
+
+/* Static description of a status code (host). */
+const char* bpt_status_str(bpt_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BPT_H */

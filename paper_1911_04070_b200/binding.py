@@ -1,0 +1,214 @@
+"""Thin Python binding of the C ABI in include/bpt.h (argument marshalling only).
+
+PyTorch supplies device memory and the current stream; every step of the path
+runs in the CUDA kernels of libbpt.so.  There is no CPU fallback: a missing
+library or a failing call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbpt.so")
+
+BPT_BIDIR, BPT_LEFT_ONLY, BPT_MODE_PAD, BPT_MODE_ALG1 = 0, 1, 0, 2
+BPT_F32, BPT_BF16 = 0, 1
+
+EXPORTS = ("bpt_graph_dims_query", "bpt_build_graph", "bpt_attn_workspace_bytes", "bpt_attn_fwd",
+           "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end")
+
+
+class BptError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (where, status_str(status), status))
+
+
+class GraphDims(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int32), ("k", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("n_levels", ctypes.c_int32), ("n_nodes", ctypes.c_int32), ("n_rel", ctypes.c_int32),
+                ("n_edges", ctypes.c_int64), ("build_workspace_bytes", ctypes.c_size_t)]
+
+
+class GraphStruct(ctypes.Structure):
+    _fields_ = [("row_ptr", ctypes.c_void_p), ("col", ctypes.c_void_p), ("rel", ctypes.c_void_p),
+                ("t_ptr", ctypes.c_void_p), ("t_dst", ctypes.c_void_p), ("t_eid", ctypes.c_void_p),
+                ("dims", GraphDims)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libbpt.so from the package directory; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libbpt.so is missing: run `python -m paper_1911_04070_b200.build` "
+                              "(there is no fallback implementation)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, u32, sz, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_float
+        lib.bpt_graph_dims_query.restype = ctypes.c_int
+        lib.bpt_graph_dims_query.argtypes = [i32, i32, u32, ctypes.POINTER(GraphDims)]
+        lib.bpt_build_graph.restype = ctypes.c_int
+        lib.bpt_build_graph.argtypes = [ctypes.POINTER(GraphDims), vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(GraphStruct)]
+        lib.bpt_attn_workspace_bytes.restype = sz
+        lib.bpt_attn_workspace_bytes.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, ctypes.c_int]
+        lib.bpt_attn_fwd.restype = ctypes.c_int
+        lib.bpt_attn_fwd.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
+                                     vp, vp, vp, sz, vp]
+        lib.bpt_attn_bwd.restype = ctypes.c_int
+        lib.bpt_attn_bwd.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
+                                     vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.bpt_trace_begin.restype = ctypes.c_int
+        lib.bpt_trace_begin.argtypes = [i32, vp]
+        lib.bpt_trace_end.restype = ctypes.c_int
+        lib.bpt_trace_end.argtypes = [ctypes.POINTER(i32), ctypes.POINTER(f32), ctypes.POINTER(ctypes.c_char_p), i32]
+        lib.bpt_status_str.restype = ctypes.c_char_p
+        lib.bpt_status_str.argtypes = [ctypes.c_int]
+        _lib = lib
+    return _lib
+
+
+def status_str(status: int) -> str:
+    return load_library().bpt_status_str(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise BptError(status, where)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return BPT_F32
+    if t.dtype == torch.bfloat16:
+        return BPT_BF16
+    raise TypeError("only float32 and bfloat16 tensors are supported, got %s" % t.dtype)
+
+
+def bpt_graph_dims_query(n: int, k: int, flags: int = 0) -> GraphDims:
+    dims = GraphDims()
+    _check(load_library().bpt_graph_dims_query(n, k, flags, ctypes.byref(dims)), "bpt_graph_dims_query")
+    return dims
+
+
+class Graph:
+    """Device-resident BPT graph: owns the index tensors the C struct points at."""
+
+    def __init__(self, dims: GraphDims, device, with_transpose: bool):
+        E, N = dims.n_edges, dims.n_nodes
+        i32 = dict(dtype=torch.int32, device=device)
+        self.dims = dims
+        self.row_ptr = torch.empty(N + 1, **i32)
+        self.col = torch.empty(E, **i32)
+        self.rel = torch.empty(E, **i32)
+        self.t_ptr = torch.empty(N + 1, **i32) if with_transpose else None
+        self.t_dst = torch.empty(E, **i32) if with_transpose else None
+        self.t_eid = torch.empty(E, **i32) if with_transpose else None
+        self.c = GraphStruct()
+
+    n = property(lambda s: s.dims.n)
+    k = property(lambda s: s.dims.k)
+    n_nodes = property(lambda s: s.dims.n_nodes)
+    n_edges = property(lambda s: s.dims.n_edges)
+    n_rel = property(lambda s: s.dims.n_rel)
+
+
+def bpt_build_graph(n: int, k: int, flags: int = 0, device="cuda", with_transpose: bool = True) -> Graph:
+    """Builds the graph of (n, k, flags) on `device` with the library's kernels."""
+    lib = load_library()
+    dims = bpt_graph_dims_query(n, k, flags)
+    device = torch.device(device)
+    with torch.cuda.device(device):
+        g = Graph(dims, device, with_transpose)
+        ws = torch.empty(max(int(dims.build_workspace_bytes), 1), dtype=torch.uint8, device=device)
+        _check(lib.bpt_build_graph(ctypes.byref(dims), _ptr(g.row_ptr), _ptr(g.col), _ptr(g.rel),
+                                   _ptr(g.t_ptr), _ptr(g.t_dst), _ptr(g.t_eid), _ptr(ws), _stream(),
+                                   ctypes.byref(g.c)), "bpt_build_graph")
+        g._build_ws = ws  # keep alive until the stream has run the build
+    return g
+
+
+def bpt_attn_workspace_bytes(g: Graph, B: int, H: int, d: int, dtype_code: int, backward: bool) -> int:
+    return int(load_library().bpt_attn_workspace_bytes(ctypes.byref(g.c), B, H, d, dtype_code, int(backward)))
+
+
+def _check_layout(g: Graph, q, *same):
+    if q.dim() != 4 or q.shape[1] != g.n_nodes:
+        raise ValueError("expected [B, n_nodes=%d, H, d], got %s" % (g.n_nodes, tuple(q.shape)))
+    for t in same:
+        if t.shape != q.shape or t.dtype != q.dtype or t.device != q.device:
+            raise ValueError("q, k, v, out, d_out must share shape, dtype and device")
+    for t in (q,) + same:
+        if not t.is_contiguous():
+            raise ValueError("tensors must be contiguous")
+        if not t.is_cuda:
+            raise ValueError("tensors must live on a CUDA device")
+
+
+def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, workspace=None):
+    """Returns (out [B,N,H,d], lse [B,N,H] fp32)."""
+    lib = load_library()
+    _check_layout(g, q, k, v)
+    B, N, H, d = q.shape
+    code = _dtype_code(q)
+    if rel_emb.shape != (g.n_rel, d) or rel_emb.dtype != q.dtype or not rel_emb.is_contiguous():
+        raise ValueError("rel_emb must be contiguous [n_rel=%d, d] of the same dtype" % g.n_rel)
+    with torch.cuda.device(q.device):
+        out = torch.empty_like(q) if out is None else out
+        lse = torch.empty((B, N, H), dtype=torch.float32, device=q.device) if lse is None else lse
+        need = bpt_attn_workspace_bytes(g, B, H, d, code, False)
+        if workspace is None and need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+        _check(lib.bpt_attn_fwd(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
+                                float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
+                                0 if workspace is None else workspace.numel(), _stream()), "bpt_attn_fwd")
+    return out, lse
+
+
+def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, workspace=None,
+                 dq=None, dk=None, dv=None, d_rel=None):
+    """Returns (dq, dk, dv [B,N,H,d], d_rel [n_rel, d] fp32)."""
+    lib = load_library()
+    _check_layout(g, q, k, v, out, d_out)
+    B, N, H, d = q.shape
+    code = _dtype_code(q)
+    with torch.cuda.device(q.device):
+        dq = torch.empty_like(q) if dq is None else dq
+        dk = torch.empty_like(q) if dk is None else dk
+        dv = torch.empty_like(q) if dv is None else dv
+        d_rel = torch.empty((g.n_rel, d), dtype=torch.float32, device=q.device) if d_rel is None else d_rel
+        need = bpt_attn_workspace_bytes(g, B, H, d, code, True)
+        if workspace is None and need:
+            workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+        _check(lib.bpt_attn_bwd(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
+                                float(scale), _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq), _ptr(dk), _ptr(dv),
+                                _ptr(d_rel), _ptr(workspace), 0 if workspace is None else workspace.numel(),
+                                _stream()), "bpt_attn_bwd")
+    return dq, dk, dv, d_rel
+
+
+def bpt_trace_begin(capacity: int):
+    """Start recording one CUDA event after every kernel the library launches."""
+    _check(load_library().bpt_trace_begin(capacity, _stream()), "bpt_trace_begin")
+
+
+def bpt_trace_end(capacity: int):
+    """Stop recording; returns [(kernel name, milliseconds), ...] in launch order."""
+    n = ctypes.c_int32(0)
+    ms = (ctypes.c_float * capacity)()
+    names = (ctypes.c_char_p * capacity)()
+    _check(load_library().bpt_trace_end(ctypes.byref(n), ms, names, capacity), "bpt_trace_end")
+    return [(names[i].decode(), float(ms[i])) for i in range(min(n.value, capacity))]

@@ -1,0 +1,123 @@
+// C-ABI entry points: argument validation and dispatch.  See include/bpt.h.
+#include "bpt_internal.cuh"
+
+using namespace bpt;
+
+static bpt_status check_problem(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype, bool backward) {
+    if (!g || !g->row_ptr || !g->col || !g->rel) return BPT_ERR_INVALID_ARG;
+    if (B < 1 || H < 1) return BPT_ERR_INVALID_ARG;
+    if (dtype != BPT_F32 && dtype != BPT_BF16) return BPT_ERR_INVALID_ARG;
+    if (d != 32 && d != 64) return BPT_ERR_UNSUPPORTED;
+    TreeParams t;
+    if (!tree_params_from_dims(g->dims, &t)) return BPT_ERR_INVALID_ARG;
+    if (g->dims.n_nodes != 2 * g->dims.n - 1 || g->dims.n_edges < g->dims.n_nodes || g->dims.n_edges >= INT32_MAX)
+        return BPT_ERR_INVALID_ARG;
+    if (backward && !(g->t_ptr && g->t_dst && g->t_eid)) return BPT_ERR_INVALID_ARG;
+    return BPT_OK;
+}
+
+extern "C" size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype, int backward) {
+    if (check_problem(g, B, H, d, dtype, false) != BPT_OK) return 0;
+    return backward ? bwd_workspace_bytes(*g, B, H, d, dtype) : fwd_workspace_bytes(*g, B, H, d, dtype);
+}
+
+extern "C" bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                   const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                   void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    const bpt_status s = check_problem(g, B, H, d, dtype, false);
+    if (s != BPT_OK) return s;
+    if (!q || !k || !v || !rel_emb || !out || !lse) return BPT_ERR_INVALID_ARG;
+    const size_t need = fwd_workspace_bytes(*g, B, H, d, dtype);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return BPT_ERR_WORKSPACE;
+    AttnProblem p{};
+    p.g = g;
+    tree_params_from_dims(g->dims, &p.tree);
+    p.B = B; p.H = H; p.d = d; p.dtype = dtype;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale;
+    p.out = out; p.lse = lse;
+    p.workspace = workspace; p.workspace_bytes = workspace_bytes;
+    p.stream = (cudaStream_t)cuda_stream;
+    return launch_fwd(p);
+}
+
+extern "C" bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                   const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                   const void* out, const float* lse, const void* d_out,
+                                   void* dq, void* dk, void* dv, float* d_rel,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    const bpt_status s = check_problem(g, B, H, d, dtype, true);
+    if (s != BPT_OK) return s;
+    if (!q || !k || !v || !rel_emb || !out || !lse || !d_out || !dq || !dk || !dv || !d_rel) return BPT_ERR_INVALID_ARG;
+    const size_t need = bwd_workspace_bytes(*g, B, H, d, dtype);
+    if (need > 0 && (!workspace || workspace_bytes < need)) return BPT_ERR_WORKSPACE;
+    AttnProblem p{};
+    p.g = g;
+    tree_params_from_dims(g->dims, &p.tree);
+    p.B = B; p.H = H; p.d = d; p.dtype = dtype;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale;
+    p.out = const_cast<void*>(out); p.lse = const_cast<float*>(lse);
+    p.d_out = d_out; p.dq = dq; p.dk = dk; p.dv = dv; p.d_rel = d_rel;
+    p.workspace = workspace; p.workspace_bytes = workspace_bytes;
+    p.stream = (cudaStream_t)cuda_stream;
+    return launch_bwd(p);
+}
+
+// ---------------------------------------------------------------------------------
+// tracing
+// ---------------------------------------------------------------------------------
+namespace {
+constexpr int kTraceMax = 4096;
+struct TraceState {
+    bool on = false;
+    int n = 0, cap = 0;
+    cudaEvent_t ev[kTraceMax];
+    const char* name[kTraceMax];
+} g_trace;
+}  // namespace
+
+void bpt::trace_mark(cudaStream_t st, const char* name) {
+    if (!g_trace.on || g_trace.n >= g_trace.cap) return;
+    cudaEventRecord(g_trace.ev[g_trace.n], st);
+    g_trace.name[g_trace.n] = name;
+    ++g_trace.n;
+}
+
+extern "C" bpt_status bpt_trace_begin(int32_t capacity, void* cuda_stream) {
+    if (g_trace.on || capacity < 1 || capacity >= kTraceMax) return BPT_ERR_INVALID_ARG;
+    for (int i = 0; i <= capacity; ++i)
+        if (cudaEventCreate(&g_trace.ev[i]) != cudaSuccess) return BPT_ERR_CUDA;
+    g_trace.cap = capacity + 1;
+    g_trace.n = 0;
+    g_trace.on = true;
+    bpt::trace_mark((cudaStream_t)cuda_stream, "begin");
+    return BPT_OK;
+}
+
+extern "C" bpt_status bpt_trace_end(int32_t* n_marks, float* ms, const char** names, int32_t capacity) {
+    if (!g_trace.on || !n_marks) return BPT_ERR_INVALID_ARG;
+    g_trace.on = false;
+    bpt_status st = BPT_OK;
+    const int n = g_trace.n - 1;  // intervals
+    if (n >= 1 && cudaEventSynchronize(g_trace.ev[n]) != cudaSuccess) st = BPT_ERR_CUDA;
+    for (int i = 0; i < n && i < capacity && st == BPT_OK; ++i) {
+        if (ms && cudaEventElapsedTime(&ms[i], g_trace.ev[i], g_trace.ev[i + 1]) != cudaSuccess) st = BPT_ERR_CUDA;
+        if (names) names[i] = g_trace.name[i + 1];
+    }
+    for (int i = 0; i < g_trace.cap; ++i) cudaEventDestroy(g_trace.ev[i]);
+    *n_marks = n < 0 ? 0 : n;
+    g_trace.n = g_trace.cap = 0;
+    return st;
+}
+
+extern "C" const char* bpt_status_str(bpt_status s) {
+    switch (s) {
+        case BPT_OK: return "ok";
+        case BPT_ERR_INVALID_ARG: return "invalid argument";
+        case BPT_ERR_UNSUPPORTED: return "unsupported size or type";
+        case BPT_ERR_WORKSPACE: return "workspace missing or too small";
+        case BPT_ERR_CUDA: return "CUDA error";
+        case BPT_ERR_TIMEOUT: return "device-side wait timed out";
+        case BPT_ERR_OVERFLOW: return "edge count exceeds 32-bit indices";
+    }
+    return "unknown status";
+}

@@ -1,0 +1,148 @@
+// Forward graph self-attention over the CSR (arXiv 1911.04070: GSA of Sec. 3.1 with the
+// relative-position term of Sec. 3.4).  General row kernel: one CTA per (batch, node,
+// head group); its warps take the row's edges in turns, each keeps an online softmax in
+// registers, and the per-warp states are merged in a fixed order through shared memory.
+#include "bpt_internal.cuh"
+#include "row_map.cuh"
+
+namespace bpt {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+template <typename T, int D, int U>
+__global__ void __launch_bounds__(256)
+fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col, const int32_t* __restrict__ rel,
+                const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
+                T* __restrict__ out, float* __restrict__ lse, int N, int H, int ngroups, float scale_log2e) {
+    using M = RowMap<T, D>;
+    constexpr int EPL = M::EPL;
+    extern __shared__ float smem[];
+    const int nw = blockDim.x >> 5, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t bid = blockIdx.x;
+    const int u = N - 1 - (int)(bid % N);  // long span rows first
+    const int hg = (int)((bid / N) % ngroups);
+    const int b = (int)(bid / ((int64_t)N * ngroups));
+    const int head = hg * M::HPW + lane / M::G;
+    const bool head_ok = head < H;
+    const int hc = head_ok ? head : H - 1;
+    const int sub = lane % M::G;
+    const size_t rs = (size_t)H * D;
+    const size_t boff = (size_t)b * N * rs + (size_t)hc * D;
+
+    float qv[EPL];
+    M::load(q + boff + (size_t)u * rs, sub, qv);
+#pragma unroll
+    for (int c = 0; c < EPL; ++c) qv[c] *= scale_log2e;
+
+    float m = -INFINITY, l = 0.f, acc[EPL];
+#pragma unroll
+    for (int c = 0; c < EPL; ++c) acc[c] = 0.f;
+
+    const int a = row_ptr[u], z = row_ptr[u + 1];
+    for (int e0 = a + w * U; e0 < z; e0 += nw * U) {
+        const int cnt = min(U, z - e0);
+        int my_c = 0, my_r = 0;
+        if (lane < cnt) { my_c = col[e0 + lane]; my_r = rel[e0 + lane]; }
+        float s[U], vv[U][EPL];
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+            const int c = __shfl_sync(0xffffffffu, my_c, j), rr = __shfl_sync(0xffffffffu, my_r, j);
+            if (j < cnt) {
+                float kk[EPL], rv[EPL];
+                M::load(k + boff + (size_t)c * rs, sub, kk);
+                M::load(r + (size_t)rr * D, sub, rv);
+                M::load(v + boff + (size_t)c * rs, sub, vv[j]);
+                float d = 0.f;
+#pragma unroll
+                for (int x = 0; x < EPL; ++x) d = fmaf(qv[x], kk[x] + rv[x], d);
+                s[j] = d;
+            } else {
+                s[j] = -INFINITY;
+#pragma unroll
+                for (int x = 0; x < EPL; ++x) vv[j][x] = 0.f;
+            }
+        }
+        float m_new = m;
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+            s[j] = M::head_sum(s[j]);
+            m_new = fmaxf(m_new, s[j]);
+        }
+        const float corr = fast_exp2(m - m_new);
+        l *= corr;
+#pragma unroll
+        for (int x = 0; x < EPL; ++x) acc[x] *= corr;
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+            const float p = fast_exp2(s[j] - m_new);
+            l += p;
+#pragma unroll
+            for (int x = 0; x < EPL; ++x) acc[x] = fmaf(p, vv[j][x], acc[x]);
+        }
+        m = m_new;
+    }
+
+    if (nw > 1) {  // merge the warps' (m, l, acc) in warp order
+        float* sm_m = smem;
+        float* sm_l = smem + nw * 32;
+        float* sm_a = smem + 2 * nw * 32;
+        sm_m[w * 32 + lane] = m;
+        sm_l[w * 32 + lane] = l;
+#pragma unroll
+        for (int x = 0; x < EPL; ++x) sm_a[(w * EPL + x) * 32 + lane] = acc[x];
+        __syncthreads();
+        if (w != 0) return;
+        float mt = -INFINITY;
+        for (int j = 0; j < nw; ++j) mt = fmaxf(mt, sm_m[j * 32 + lane]);
+        l = 0.f;
+#pragma unroll
+        for (int x = 0; x < EPL; ++x) acc[x] = 0.f;
+        for (int j = 0; j < nw; ++j) {
+            const float f = fast_exp2(sm_m[j * 32 + lane] - mt);
+            l = fmaf(sm_l[j * 32 + lane], f, l);
+#pragma unroll
+            for (int x = 0; x < EPL; ++x) acc[x] = fmaf(sm_a[(j * EPL + x) * 32 + lane], f, acc[x]);
+        }
+        m = mt;
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+    for (int x = 0; x < EPL; ++x) acc[x] *= inv;
+    if (head_ok) {
+        M::store(out + boff + (size_t)u * rs, sub, acc);
+        if (sub == 0) lse[((size_t)b * N + u) * H + head] = (m + log2f(l)) * kLn2;
+    }
+}
+
+int rows_kernel_warps(const bpt_graph& g) {
+    const double avg = (double)g.dims.n_edges / (double)g.dims.n_nodes;
+    return avg >= 96.0 ? 8 : (avg >= 24.0 ? 4 : 2);
+}
+
+template <typename T, int D>
+static bpt_status launch_rows(const AttnProblem& p) {
+    using M = RowMap<T, D>;
+    constexpr int U = 4;
+    const bpt_graph& g = *p.g;
+    const int N = g.dims.n_nodes;
+    const int ngroups = (p.H + M::HPW - 1) / M::HPW;
+    const int nw = rows_kernel_warps(g);
+    const int64_t blocks = (int64_t)p.B * N * ngroups;
+    if (blocks > 0x7fffffffll) return BPT_ERR_UNSUPPORTED;
+    const size_t smem = nw > 1 ? (size_t)nw * 32 * (2 + M::EPL) * sizeof(float) : 0;
+    fwd_rows_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem, p.stream>>>(
+        g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
+        (T*)p.out, p.lse, N, p.H, ngroups, p.scale * kLog2e);
+    trace_mark(p.stream, "fwd_rows");
+    return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
+}
+
+size_t fwd_workspace_bytes(const bpt_graph&, int, int, int, bpt_dtype) { return 0; }
+
+bpt_status launch_fwd(const AttnProblem& p) {
+    if (p.dtype == BPT_F32) return p.d == 64 ? launch_rows<float, 64>(p) : launch_rows<float, 32>(p);
+    return p.d == 64 ? launch_rows<__nv_bfloat16, 64>(p) : launch_rows<__nv_bfloat16, 32>(p);
+}
+
+}  // namespace bpt

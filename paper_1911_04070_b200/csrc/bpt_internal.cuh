@@ -1,0 +1,43 @@
+// Declarations shared by the translation units of libbpt (not part of the C ABI).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/bpt.h"
+#include "bpt_tree.cuh"
+
+namespace bpt {
+
+bool tree_params_from_dims(const bpt_graph_dims& d, TreeParams* t);
+
+// Problem description handed to the attention launchers (all pointers device).
+struct AttnProblem {
+    const bpt_graph* g;
+    TreeParams tree;
+    int B, H, d;
+    bpt_dtype dtype;
+    const void *q, *k, *v, *rel_emb;
+    float scale;
+    // forward outputs / backward inputs
+    void* out;
+    float* lse;
+    // backward only
+    const void* d_out;
+    void *dq, *dk, *dv;
+    float* d_rel;
+    void* workspace;
+    size_t workspace_bytes;
+    cudaStream_t stream;
+};
+
+// Optional per-launch timing (see bpt_trace_begin): a mark after every kernel launch.
+void trace_mark(cudaStream_t st, const char* name);
+
+size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype);
+size_t bwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype);
+bpt_status launch_fwd(const AttnProblem& p);
+bpt_status launch_bwd(const AttnProblem& p);
+
+}  // namespace bpt

@@ -1,0 +1,31 @@
+"""Helpers shared by the GPU parity tests: tolerances and oracle drivers."""
+import numpy as np
+
+# Tolerances: max relative error against the fp64 oracle, 1e-5 for fp32 inputs and 2e-2 for
+# bf16 inputs with fp32 accumulation (outputs are rounded once to the input type).
+TOL = {"fp32": 1e-5, "bf16": 2e-2}
+
+
+def assert_close(name, got, want, tol):
+    """Both criteria: ||x-y||_inf / ||y||_inf <= tol and, element-wise,
+    |x-y| <= tol * (|y| + rms(y))."""
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    assert got.shape == want.shape, (name, got.shape, want.shape)
+    assert np.isfinite(got).all(), name + ": non-finite values"
+    err = np.abs(got - want)
+    scale = np.abs(want).max()
+    assert scale > 0, name + ": reference is all zero"
+    rel = err.max() / scale
+    assert rel <= tol, "%s: max-norm relative error %.3e > %.1e" % (name, rel, tol)
+    rms = np.sqrt(np.mean(want * want))
+    bad = err > tol * (np.abs(want) + rms)
+    assert not bad.any(), "%s: %d elements outside tol, worst abs err %.3e (rms %.3e)" % (name, int(bad.sum()), err[bad].max(), rms)
+    return rel
+
+
+def assert_small(name, got, ref_scale, tol):
+    """For quantities that are exactly zero in theory (gradient of the ancestor relations)."""
+    got = np.asarray(got, dtype=np.float64)
+    assert np.isfinite(got).all(), name
+    assert np.abs(got).max() <= tol * ref_scale, "%s: %.3e vs scale %.3e" % (name, np.abs(got).max(), ref_scale)

@@ -1,0 +1,152 @@
+"""GPU attention forward/backward vs the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+
+from parity import TOL, assert_close, assert_small
+
+pytestmark = pytest.mark.gpu
+
+
+def _torch_inputs(x, bf16, device="cuda:0"):
+    import torch
+    dt = torch.bfloat16 if bf16 else torch.float32
+    return {name: torch.from_numpy(a).to(device=device, dtype=dt) for name, a in x.items()}
+
+
+def _np(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def run_case(n, k, flags, B, H, d, bf16, seed, std_qkv, backward=True, oracle_batches=None, std_rel=0.02):
+    """Runs the library on the full problem and the oracle (C twin) on the same inputs.
+    Returns nothing; asserts parity."""
+    import torch
+    from oracle import ctwin
+    from paper_1911_04070_b200 import binding, synth
+    tol = TOL["bf16" if bf16 else "fp32"]
+    ref = ctwin.CGraph(n, k, flags)
+    x = synth.make_inputs(B, ref.n_nodes, H, d, ref.n_rel, seed=seed, std_qkv=std_qkv, std_rel=std_rel, bf16=bf16, with_grad=backward)
+    scale = 1.0 / np.sqrt(d)
+    g = binding.bpt_build_graph(n, k, flags, device="cuda:0", with_transpose=backward)
+    t = _torch_inputs(x, bf16)
+    out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale)
+    torch.cuda.synchronize()
+    o_ref, lse_ref = ctwin.attn_fwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], scale)
+    assert_close("out", _np(out), o_ref, tol)
+    assert_close("lse", _np(lse), lse_ref, tol)
+    if not backward:
+        return
+    dq, dk, dv, dr = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"])
+    torch.cuda.synchronize()
+    rq, rk, rv, rr = ctwin.attn_bwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], scale, x["d_out"])
+    assert_close("dq", _np(dq), rq, tol)
+    assert_close("dk", _np(dk), rk, tol)
+    assert_close("dv", _np(dv), rv, tol)
+    L, W = ref.L, k + 1
+    first_anc = 1 + 2 * L * W
+    assert_close("d_rel", _np(dr)[:first_anc], rr[:first_anc], tol)
+    assert_small("d_rel[anc]", _np(dr)[first_anc:], np.abs(rr).max(), tol)
+    # atomics-free, fixed order: a second run gives the same bits
+    dq2, dk2, dv2, dr2 = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"])
+    out2, lse2 = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale)
+    torch.cuda.synchronize()
+    for a, b in ((dq, dq2), (dk, dk2), (dv, dv2), (dr, dr2), (out, out2), (lse, lse2)):
+        assert torch.equal(a, b)
+
+
+SMALL = [
+    # n, k, flags, B, H, d, bf16
+    (2, 1, 0, 1, 1, 32, False),
+    (8, 1, 0, 2, 1, 32, False),
+    (16, 2, 1, 2, 3, 64, False),       # H not a multiple of the heads per warp
+    (64, 3, 0, 3, 5, 32, True),
+    (64, 70, 0, 2, 2, 64, True),       # k >= n: dense token rows
+    (128, 5, 2, 2, 8, 64, True),       # Algorithm-1 graph
+    (256, 4, 0, 2, 9, 64, True),       # 9 heads: two head groups for bf16
+    (512, 16, 1, 1, 4, 64, False),
+    (1024, 1, 0, 1, 8, 32, True),
+    (2048, 3, 3, 1, 2, 64, True),
+]
+
+
+@pytest.mark.parametrize("n,k,flags,B,H,d,bf16", SMALL)
+def test_small_cases(n, k, flags, B, H, d, bf16):
+    run_case(n, k, flags, B, H, d, bf16, seed=100 + n + k, std_qkv=1.0 if not bf16 else 0.5, std_rel=0.3)
+
+
+def test_against_numpy_oracle_directly():
+    import torch
+    from oracle import bpt_oracle as orc
+    from paper_1911_04070_b200 import binding, synth
+    n, k, B, H, d = 32, 2, 2, 2, 32
+    ref = orc.enumerate_graph(n, k, 0)
+    x = synth.make_inputs(B, ref.n_nodes, H, d, ref.n_rel, seed=9, std_qkv=1.0, std_rel=0.5, bf16=False)
+    g = binding.bpt_build_graph(n, k, 0, device="cuda:0")
+    t = _torch_inputs(x, False)
+    out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.25)
+    grads = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.25, out, lse, t["d_out"])
+    o_ref, lse_ref = orc.attn_fwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], 0.25)
+    refs = orc.attn_bwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], 0.25, x["d_out"])
+    assert_close("out", _np(out), o_ref, 1e-5)
+    assert_close("lse", _np(lse), lse_ref, 1e-5)
+    first_anc = 1 + 2 * ref.L * (k + 1)
+    for name, a, b in zip(("dq", "dk", "dv"), grads[:3], refs[:3]):
+        assert_close(name, _np(a), b, 1e-5)
+    assert_close("d_rel", _np(grads[3])[:first_anc], refs[3][:first_anc], 1e-5)
+
+
+def _cfg(name):
+    from paper_1911_04070_b200 import synth
+    c = dict(synth.CONFIGS[name])
+    return c
+
+
+def test_config1_tiny_fp32():
+    c = _cfg("cfg1_tiny")
+    run_case(c["n"], c["k"], c["flags"], c["B"], c["H"], c["d"], c["bf16"], c["seed"], c["std_qkv"], c["backward"])
+
+
+def test_config2_classification_forward():
+    c = _cfg("cfg2_cls")
+    run_case(c["n"], c["k"], c["flags"], c["B"], c["H"], c["d"], c["bf16"], c["seed"], c["std_qkv"], c["backward"])
+
+
+def test_config3_document_translation():
+    c = _cfg("cfg3_doc_mt")
+    run_case(c["n"], c["k"], c["flags"], c["B"], c["H"], c["d"], c["bf16"], c["seed"], c["std_qkv"], c["backward"])
+
+
+def test_config4_char_lm_full_size():
+    c = _cfg("cfg4_char_lm")
+    run_case(c["n"], c["k"], c["flags"], c["B"], c["H"], c["d"], c["bf16"], c["seed"], c["std_qkv"], c["backward"])
+
+
+@pytest.mark.parametrize("n,k", [(1024, 4), (4096, 16), (16384, 4), (65536, 16)])
+def test_config5_sweep_points(n, k):
+    from paper_1911_04070_b200 import synth
+    c = synth.sweep_configs()["cfg5_n%d_k%d" % (n, k)]
+    # the oracle covers two batch entries' worth of work per point; the library runs that same problem
+    run_case(c["n"], c["k"], c["flags"], min(c["B"], 2), c["H"], c["d"], c["bf16"], c["seed"], c["std_qkv"], True)
+
+
+def test_argument_errors_do_not_launch():
+    import ctypes
+    import torch
+    from paper_1911_04070_b200 import binding
+    g = binding.bpt_build_graph(64, 2, 0, device="cuda:0", with_transpose=False)
+    q = torch.zeros((1, g.n_nodes, 2, 48), device="cuda:0")
+    r = torch.zeros((g.n_rel, 48), device="cuda:0")
+    with pytest.raises(binding.BptError) as ei:      # head size 48 is not supported
+        binding.bpt_attn_fwd(g, q, q, q, r, 1.0)
+    assert ei.value.status == 2
+    q = torch.zeros((1, g.n_nodes, 2, 64), device="cuda:0")
+    r = torch.zeros((g.n_rel, 64), device="cuda:0")
+    out, lse = binding.bpt_attn_fwd(g, q, q, q, r, 1.0)
+    with pytest.raises(binding.BptError) as ei:      # backward needs the by-source lists
+        binding.bpt_attn_bwd(g, q, q, q, r, 1.0, out, lse, q)
+    assert ei.value.status == 1
+    g2 = binding.bpt_build_graph(64, 2, 0, device="cuda:0")
+    ws = torch.empty(16, dtype=torch.uint8, device="cuda:0")
+    with pytest.raises(binding.BptError) as ei:      # undersized workspace
+        binding.bpt_attn_bwd(g2, q, q, q, r, 1.0, out, lse, q, workspace=ws)
+    assert ei.value.status == 3
