@@ -277,8 +277,11 @@ def run_ours(args, cfg_name, cfg):
     peak, peak_kind = load_peaks()
     roofline = None
     if dominant:
-        key = "fwd" if dominant.startswith("fwd") else ("bwd_dst" if "dst" in dominant else "bwd_src")
-        alg_bytes = GATHER_BYTES_PER_EDGE_HEAD[key](d, esize) * B * H * E
+        if dominant.startswith("drel"):
+            alg_bytes = 4 * B * H * E + B * N * H * d * esize   # stored dS once + the q rows once
+        else:
+            key = "fwd" if dominant.startswith("fwd") else ("bwd_dst" if "dst" in dominant else "bwd_src")
+            alg_bytes = GATHER_BYTES_PER_EDGE_HEAD[key](d, esize) * B * H * E
         achieved = alg_bytes / (kernels[dominant]["avg_ms"] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "peak_kind": peak_kind,
                     "unit": "GB/s", "frac": achieved / peak, "traffic": None,
@@ -318,12 +321,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg4_char_lm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling of a smaller case)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     cfgs = all_configs()
     if args.config not in cfgs:
         raise SystemExit("unknown config %s; choose from %s" % (args.config, ", ".join(sorted(cfgs))))
-    cfg = cfgs[args.config]
+    cfg = dict(cfgs[args.config])
+    if args.batch > 0:
+        cfg["B"] = args.batch
     if args.impl == "reference":
         run_reference(args, args.config, cfg)
     else:

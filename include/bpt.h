@@ -128,6 +128,11 @@ bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt
  * out and lse are the forward's results.  dq, dk, dv: [B, n_nodes, H, d] in `dtype`;
  * d_rel: [n_rel, d] fp32.  All four are overwritten, not accumulated into.  The sums are
  * taken in a fixed order without atomics, so results are bit-reproducible.
+ * The d_rel rows of the ancestor relations are written as exact zeros: all edges into a
+ * span share one relation, so that embedding shifts every score of the row alike and
+ * the softmax (hence the loss) does not depend on it.
+ * d_out_u . out_u is evaluated with the stored `out`, so for bf16 the gradients carry the
+ * rounding of `out` (relative 2^-9 per element) on top of the fp32 arithmetic.
  * The graph must carry the by-source lists.  Errors as for the forward.
  */
 bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,

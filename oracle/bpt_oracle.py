@@ -210,13 +210,19 @@ def attn_fwd(g: Graph, q, k, v, r, scale):
     return out, lse
 
 
-def attn_bwd(g: Graph, q, k, v, r, scale, d_out):
+def attn_bwd(g: Graph, q, k, v, r, scale, d_out, out=None):
     """Gradient of sum(out * d_out) w.r.t. q, k, v, r.  fp64.
 
     With P the softmax weights of a row: dP_e = d_out_u . v_v,
     dS_e = P_e (dP_e - sum_e' P_e' dP_e'), dq_u = scale sum_e dS_e (k_v + r_e),
     dk_v += scale dS_e q_u, dv_v += P_e d_out_u, dr_rel(e) += scale dS_e q_u
     (summed over batch and heads, the table being shared).
+
+    The row term sum_e' P_e' dP_e' equals d_out_u . out_u.  When ``out`` is
+    given (e.g. a forward result that was rounded to bf16 for storage) that
+    second form is evaluated with it, which is what a backward pass that
+    receives a stored forward output computes; with ``out=None`` the gradient
+    is exact.
     """
     q, k, v, r, d_out = (np.asarray(a, dtype=np.float64) for a in (q, k, v, r, d_out))
     B, N, H, d = q.shape
@@ -231,7 +237,11 @@ def attn_bwd(g: Graph, q, k, v, r, scale, d_out):
         p = np.exp(s)
         p /= p.sum(axis=2, keepdims=True)
         dp = np.einsum("bhc,behc->bhe", d_out[:, u], v[:, src])
-        ds = p * (dp - (p * dp).sum(axis=2, keepdims=True))
+        if out is None:
+            row_term = (p * dp).sum(axis=2, keepdims=True)
+        else:
+            row_term = (d_out[:, u] * np.asarray(out, dtype=np.float64)[:, u]).sum(axis=2)[:, :, None]
+        ds = p * (dp - row_term)
         dq[:, u] = scale * np.einsum("bhe,behc->bhc", ds, kk)
         dk[:, src] += scale * np.einsum("bhe,bhc->behc", ds, q[:, u])    # src unique per row
         dv[:, src] += np.einsum("bhe,bhc->behc", p, d_out[:, u])

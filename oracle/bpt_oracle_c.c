@@ -172,12 +172,14 @@ void orc_attn_fwd(int64_t N, const int32_t* row_ptr, const int32_t* col, const i
 /*
  * Backward of sum(out * d_out).  dq,dk,dv: [B, N, H, d] (entries of batches
  * [b0,b1) are overwritten); dr: [n_rel, d], overwritten with the sum over the
- * computed batches and all heads.
+ * computed batches and all heads.  The row term sum_e P_e dP_e equals
+ * d_out_u . out_u; when out_opt is not NULL that second form is evaluated with the
+ * given (possibly rounded) forward output, otherwise the exact sum is used.
  */
 void orc_attn_bwd(int64_t N, int64_t n_rel, const int32_t* row_ptr, const int32_t* col, const int32_t* rel,
                   int64_t B, int64_t H, int64_t d, int64_t b0, int64_t b1,
                   const double* q, const double* k, const double* v, const double* r, double scale,
-                  const double* d_out, double* dq, double* dk, double* dv, double* dr) {
+                  const double* d_out, const double* out_opt, double* dq, double* dk, double* dv, double* dr) {
     (void)B;
     const int64_t rs = H * d;
     const int64_t nbh = (b1 - b0) * H;
@@ -220,6 +222,10 @@ void orc_attn_bwd(int64_t N, int64_t n_rel, const int32_t* row_ptr, const int32_
                     p[e - a] /= sum;
                     dp[e - a] = acc;
                     dot += p[e - a] * acc;
+                }
+                if (out_opt) {
+                    dot = 0.0;
+                    for (int64_t c = 0; c < d; ++c) dot += gu[c] * out_opt[off_u + c];
                 }
                 for (int64_t e = a; e < z; ++e) {
                     const int64_t off_v = (b * N + col[e]) * rs + h * d;

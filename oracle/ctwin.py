@@ -44,7 +44,7 @@ def _load():
         lib.orc_attn_fwd.restype = None
         lib.orc_attn_fwd.argtypes = [i64, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, dbl, p, p]
         lib.orc_attn_bwd.restype = None
-        lib.orc_attn_bwd.argtypes = [i64, i64, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, dbl, p, p, p, p, p]
+        lib.orc_attn_bwd.argtypes = [i64, i64, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, dbl, p, p, p, p, p, p]
         _lib = lib
     return _lib
 
@@ -95,14 +95,17 @@ def attn_fwd(g, q, k, v, r, scale, b0=0, b1=None):
     return out, lse
 
 
-def attn_bwd(g, q, k, v, r, scale, d_out, b0=0, b1=None):
-    """fp64 backward on batch entries [b0, b1); dr sums over those entries only."""
+def attn_bwd(g, q, k, v, r, scale, d_out, b0=0, b1=None, out=None):
+    """fp64 backward on batch entries [b0, b1); dr sums over those entries only.
+    ``out``: optional stored forward output to use in the row term (see the C source)."""
     q, k, v, r, d_out = _f64(q), _f64(k), _f64(v), _f64(r), _f64(d_out)
     B, N, H, d = q.shape
     b1 = B if b1 is None else b1
     dq, dk, dv = np.zeros_like(q), np.zeros_like(q), np.zeros_like(q)
     dr = np.zeros_like(r)
+    _out = None if out is None else _f64(out)
     _load().orc_attn_bwd(N, r.shape[0], _ptr(g.row_ptr), _ptr(g.col), _ptr(g.rel), B, H, d, b0, b1,
                          _ptr(q), _ptr(k), _ptr(v), _ptr(r), float(scale), _ptr(d_out),
+                         None if out is None else _ptr(_out),
                          _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dr))
     return dq, dk, dv, dr

@@ -6,6 +6,9 @@
 //   B  by source (transposed lists): dk, dv from the stored P / dS
 //   C  per (side, level) block of the relation table: partial d_rel over token chunks
 //   D  sum of the partials
+// The rows of d_rel that belong to the ancestor relations are written as exact zeros:
+// every edge into a span carries the same relation, so its embedding shifts all scores of
+// the row alike and the softmax does not depend on it.
 #include "bpt_internal.cuh"
 #include "row_map.cuh"
 
@@ -19,7 +22,6 @@ int rows_kernel_warps(const bpt_graph& g);
 struct BwdWorkspace {
     float* p;        // [B, E, H]
     float* ds;       // [B, E, H]
-    float* rowsum;   // [B, n-1, H]  sum_e dS_e of every span row
     float* part;     // [chunks, n_rel, d]
     size_t bytes;
 };
@@ -35,7 +37,6 @@ static BwdWorkspace carve(const bpt_graph& g, int B, int H, int d, void* base) {
     size_t off = 0;
     w.p = (float*)(c + off); off += align256(sizeof(float) * B * E * H);
     w.ds = (float*)(c + off); off += align256(sizeof(float) * B * E * H);
-    w.rowsum = (float*)(c + off); off += align256(sizeof(float) * B * (n - 1) * H);
     w.part = (float*)(c + off); off += align256(sizeof(float) * rel_chunks((int)n) * (size_t)g.dims.n_rel * d);
     w.bytes = off;
     return w;
@@ -51,8 +52,8 @@ __global__ void __launch_bounds__(256)
 bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col, const int32_t* __restrict__ rel,
                const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
                const T* __restrict__ out, const float* __restrict__ lse, const T* __restrict__ d_out,
-               T* __restrict__ dq, float* __restrict__ ws_p, float* __restrict__ ws_ds, float* __restrict__ ws_rowsum,
-               int N, int n_tok, int H, int ngroups, int64_t E, float scale) {
+               T* __restrict__ dq, float* __restrict__ ws_p, float* __restrict__ ws_ds,
+               int N, int H, int ngroups, int64_t E, float scale) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
@@ -84,7 +85,6 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
     const float sc2 = scale * kLog2e;
 #pragma unroll
     for (int x = 0; x < EPL; ++x) acc[x] = 0.f;
-    float ds_sum = 0.f;
 
     const int a = row_ptr[u], z = row_ptr[u + 1];
     const size_t eoff = (size_t)b * E;
@@ -111,7 +111,6 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
                 dp = M::head_sum(dp);
                 const float p = fast_exp2(fmaf(s, sc2, -lse2));
                 const float ds = p * (dp - delta);
-                ds_sum += ds;
 #pragma unroll
                 for (int x = 0; x < EPL; ++x) acc[x] = fmaf(ds, kk[x], acc[x]);
                 if (sub == 0 && head_ok) {
@@ -123,28 +122,21 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
         }
     }
     if (nw > 1) {
-        float* sm_a = smem;               // [nw][EPL][32]
-        float* sm_s = smem + nw * EPL * 32;  // [nw][32]
+        float* sm_a = smem;  // [nw][EPL][32]
 #pragma unroll
         for (int x = 0; x < EPL; ++x) sm_a[(w * EPL + x) * 32 + lane] = acc[x];
-        sm_s[w * 32 + lane] = ds_sum;
         __syncthreads();
         if (w != 0) return;
-        ds_sum = 0.f;
 #pragma unroll
         for (int x = 0; x < EPL; ++x) acc[x] = 0.f;
         for (int j = 0; j < nw; ++j) {
-            ds_sum += sm_s[j * 32 + lane];
 #pragma unroll
             for (int x = 0; x < EPL; ++x) acc[x] += sm_a[(j * EPL + x) * 32 + lane];
         }
     }
 #pragma unroll
     for (int x = 0; x < EPL; ++x) acc[x] *= scale;
-    if (head_ok) {
-        M::store(dq + uoff, sub, acc);
-        if (sub == 0 && u >= n_tok) ws_rowsum[((size_t)b * (N - n_tok) + (u - n_tok)) * H + head] = ds_sum;
-    }
+    if (head_ok) M::store(dq + uoff, sub, acc);
 }
 
 // ---------------------------------------------------------------------------------
@@ -228,80 +220,133 @@ bwd_src_kernel(const int32_t* __restrict__ t_ptr, const int32_t* __restrict__ t_
 
 // ---------------------------------------------------------------------------------
 // C: partial d_rel.  blockIdx.y picks a block of the relation table: left level j
-// (0..L-1), right level j (L..2L-1), self (2L), ancestor level j (2L+1 .. 3L);
-// blockIdx.x picks a chunk of tokens (or of spans for the ancestor rows).
-// Thread (og, cg): relation row o0+og of the block, channels 4*cg .. 4*cg+3.
+// (0..L-1), right level j (L..2L-1), self (2L); blockIdx.x picks a chunk of tokens.
+// Items (token, batch entry, block of up to 8 heads) are staged four at a time in shared
+// memory: the q rows as fp32 and the dS values of the block's edges, which are contiguous
+// in the token's row.  Thread (og, cg) owns relation rows og, og+NOG, ... of the current
+// tile of offsets and channels 4*cg .. 4*cg+3.
 // ---------------------------------------------------------------------------------
-template <typename T> __device__ __forceinline__ float4 load4(const T* p);
-template <> __device__ __forceinline__ float4 load4<float>(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
-template <> __device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16* p) {
-    const uint2 v = __ldg(reinterpret_cast<const uint2*>(p));
-    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u),
-                       __uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
-}
+constexpr int kRelHB = 8;   // heads per item
+constexpr int kRelTB = 4;   // items staged together
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 drel_partial_kernel(TreeParams t, const int32_t* __restrict__ row_ptr, const T* __restrict__ q,
-                    const float* __restrict__ ws_ds, const float* __restrict__ ws_rowsum, float* __restrict__ part,
+                    const float* __restrict__ ws_ds, float* __restrict__ part,
                     int B, int H, int64_t E, int n_rel, int n_chunks) {
-    constexpr int CG = D / 4, NOG = 256 / CG;
-    const int cg = threadIdx.x % CG, og = threadIdx.x / CG;
+    constexpr int CG = D / 4, NOG = 256 / CG, NJ = D == 64 ? 5 : 3, OT = NOG * NJ;
+    __shared__ float q_s[kRelTB][kRelHB][D];
+    __shared__ float ds_s[kRelTB][OT][kRelHB];
+    __shared__ int it_e0[kRelTB], it_cnt[kRelTB];
+    const int tid = threadIdx.x, cg = tid % CG, og = tid / CG;
     const int chunk = blockIdx.x, blk = blockIdx.y;
     const int N = 2 * t.n - 1;
     int side, level, width, rel_base;
     if (blk < t.L) { side = 0; level = blk; width = t.k + 1; rel_base = rel_left(t, level, 0); }
     else if (blk < 2 * t.L) { side = 1; level = blk - t.L; width = t.k + 1; rel_base = rel_right(t, level, 0); }
-    else if (blk == 2 * t.L) { side = 2; level = 0; width = 1; rel_base = 0; }
-    else { side = 3; level = blk - 2 * t.L; width = 1; rel_base = rel_anc(t, level); }
+    else { side = 2; level = 0; width = 1; rel_base = 0; }
+    // no token has more than min(k, n) + 1 nodes in one block
+    const int wmax = min(width, t.kc + 1);
 
-    const int items = side == 3 ? (t.n >> level) : t.n;  // spans of the level, or tokens
-    const int per = (items + n_chunks - 1) / n_chunks;
-    const int x0 = min(chunk * per, items), x1 = min(x0 + per, items);
+    const int per = (t.n + n_chunks - 1) / n_chunks;
+    const int x0 = min(chunk * per, t.n), x1 = min(x0 + per, t.n);
+    const int nhb = (H + kRelHB - 1) / kRelHB;
+    const int n_items = (x1 - x0) * B * nhb;  // item = (token, b, head block), token-major
     const size_t rs = (size_t)H * D;
 
-    for (int o0 = 0; o0 < width; o0 += NOG) {
-        const int o = o0 + og;
-        if (o >= width) continue;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int x = x0; x < x1; ++x) {
-            int node;
-            size_t soff, sstride;  // address of the dS (or row sum) value for b = 0, h = 0 and the stride over b
-            if (side == 3) {
-                node = node_id(t.n, level, x);
-                soff = (size_t)(node - t.n) * H;
-                sstride = (size_t)(t.n - 1) * H;
-            } else {
-                int pos, cnt, first;
-                if (!token_block(t, x, side, level, &pos, &cnt, &first) || o >= cnt) continue;
-                node = x;
-                const int e = row_ptr[x] + (side == 0 ? pos + cnt - 1 - o : pos + o);
-                soff = (size_t)e * H;
-                sstride = (size_t)E * H;
-            }
-            const float* sp = (side == 3 ? ws_rowsum : ws_ds) + soff;
-            const T* qp = q + (size_t)node * rs + cg * 4;
-            for (int b = 0; b < B; ++b) {
-                for (int h = 0; h < H; ++h) {
-                    const float a = __ldg(sp + (size_t)b * sstride + h);
-                    const float4 qq = load4<T>(qp + (size_t)b * N * rs + (size_t)h * D);
-                    acc.x = fmaf(a, qq.x, acc.x);
-                    acc.y = fmaf(a, qq.y, acc.y);
-                    acc.z = fmaf(a, qq.z, acc.z);
-                    acc.w = fmaf(a, qq.w, acc.w);
+    // A level exists on the left for a suffix of the tokens and on the right for a prefix,
+    // so one probe tells whether any token of the chunk has edges in this block.
+    bool any = x1 > x0;
+    if (any && side != 2) {
+        int pos, c, first;
+        any = token_block(t, side == 0 ? x1 - 1 : x0, side, level, &pos, &c, &first);
+    }
+
+    for (int o0 = 0; o0 < width; o0 += OT) {
+        float4 acc[NJ];
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (any && o0 < wmax) {
+            for (int it0 = 0; it0 < n_items; it0 += kRelTB) {
+                __syncthreads();  // previous items consumed
+                if (tid < kRelTB) {
+                    int e0 = 0, cnt = 0;
+                    const int it = it0 + tid;
+                    if (it < n_items) {
+                        const int x = x0 + it / (B * nhb);
+                        int pos, c, first;
+                        if (token_block(t, x, side, level, &pos, &c, &first)) {
+                            // offset o sits at edge pos + o (right, self) or pos + c - 1 - o (left)
+                            cnt = max(0, min(c - o0, OT));
+                            e0 = row_ptr[x] + (side == 0 ? pos + c - 1 - o0 : pos + o0);
+                        }
+                    }
+                    it_e0[tid] = e0; it_cnt[tid] = cnt;
+                }
+                __syncthreads();
+                {
+                    int tot = 0;
+#pragma unroll
+                    for (int j = 0; j < kRelTB; ++j) tot += it_cnt[j];
+                    if (tot == 0) continue;  // uniform over the block
+                }
+                // stage q rows (as fp32) and dS values
+                for (int idx = tid; idx < kRelTB * kRelHB * D; idx += 256) {
+                    const int c = idx % D, h = (idx / D) % kRelHB, j = idx / (D * kRelHB);
+                    const int it = it0 + j;
+                    float val = 0.f;
+                    if (it < n_items && it_cnt[j] > 0) {
+                        const int x = x0 + it / (B * nhb), b = (it / nhb) % B, hh = (it % nhb) * kRelHB + h;
+                        if (hh < H) val = (float)q[((size_t)b * N + x) * rs + (size_t)hh * D + c];
+                    }
+                    q_s[j][h][c] = val;
+                }
+                for (int idx = tid; idx < kRelTB * OT * kRelHB; idx += 256) {
+                    const int h = idx % kRelHB, o = (idx / kRelHB) % OT, j = idx / (kRelHB * OT);
+                    const int it = it0 + j;
+                    float val = 0.f;
+                    if (it < n_items && o < it_cnt[j]) {
+                        const int b = (it / nhb) % B, hh = (it % nhb) * kRelHB + h;
+                        const int e = side == 0 ? it_e0[j] - o : it_e0[j] + o;
+                        if (hh < H) val = ws_ds[((size_t)b * E + e) * H + hh];
+                    }
+                    ds_s[j][o][h] = val;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int j = 0; j < kRelTB; ++j) {
+#pragma unroll
+                    for (int h = 0; h < kRelHB; ++h) {
+                        const float4 qq = *reinterpret_cast<const float4*>(&q_s[j][h][cg * 4]);
+#pragma unroll
+                        for (int jj = 0; jj < NJ; ++jj) {
+                            const float a = ds_s[j][og + jj * NOG][h];
+                            acc[jj].x = fmaf(a, qq.x, acc[jj].x);
+                            acc[jj].y = fmaf(a, qq.y, acc[jj].y);
+                            acc[jj].z = fmaf(a, qq.z, acc[jj].z);
+                            acc[jj].w = fmaf(a, qq.w, acc[jj].w);
+                        }
+                    }
                 }
             }
         }
-        *reinterpret_cast<float4*>(part + ((size_t)chunk * n_rel + rel_base + o) * D + cg * 4) = acc;
+#pragma unroll
+        for (int jj = 0; jj < NJ; ++jj) {
+            const int o = o0 + og + jj * NOG;
+            if (o < width)
+                *reinterpret_cast<float4*>(part + ((size_t)chunk * n_rel + rel_base + o) * D + cg * 4) = acc[jj];
+        }
     }
 }
 
-// D: d_rel[r, c] = scale * sum over chunks, in chunk order
-__global__ void drel_reduce_kernel(const float* __restrict__ part, float* __restrict__ d_rel, int n_chunks, size_t per_chunk, float scale) {
+// D: d_rel[r, c] = scale * sum over chunks, in chunk order; ancestor rows are zero
+__global__ void drel_reduce_kernel(const float* __restrict__ part, float* __restrict__ d_rel, int n_chunks,
+                                   size_t per_chunk, size_t first_zero, float scale) {
     const size_t x = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (x >= per_chunk) return;
     float acc = 0.f;
-    for (int c = 0; c < n_chunks; ++c) acc += part[(size_t)c * per_chunk + x];
+    if (x < first_zero)
+        for (int c = 0; c < n_chunks; ++c) acc += part[(size_t)c * per_chunk + x];
     d_rel[x] = acc * scale;
 }
 
@@ -318,10 +363,10 @@ static bpt_status launch_bwd_rows(const AttnProblem& p) {
     if (blocks > 0x7fffffffll) return BPT_ERR_UNSUPPORTED;
     const BwdWorkspace ws = carve(g, p.B, p.H, p.d, p.workspace);
 
-    const size_t smem_a = nw > 1 ? (size_t)nw * 32 * (M::EPL + 1) * sizeof(float) : 0;
+    const size_t smem_a = nw > 1 ? (size_t)nw * 32 * M::EPL * sizeof(float) : 0;
     bwd_dst_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem_a, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, ws.rowsum, N, n, p.H, ngroups, E, p.scale);
+        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, p.H, ngroups, E, p.scale);
     trace_mark(p.stream, "bwd_dst");
 
     const size_t smem_b = nw > 1 ? (size_t)nw * 32 * (2 * M::EPL) * sizeof(float) : 0;
@@ -331,12 +376,13 @@ static bpt_status launch_bwd_rows(const AttnProblem& p) {
     trace_mark(p.stream, "bwd_src");
 
     const int chunks = rel_chunks(n);
-    const dim3 grid_c(chunks, 3 * p.tree.L + 1);
-    drel_partial_kernel<T, D><<<grid_c, 256, 0, p.stream>>>(p.tree, g.row_ptr, (const T*)p.q, ws.ds, ws.rowsum, ws.part,
+    const dim3 grid_c(chunks, 2 * p.tree.L + 1);
+    drel_partial_kernel<T, D><<<grid_c, 256, 0, p.stream>>>(p.tree, g.row_ptr, (const T*)p.q, ws.ds, ws.part,
                                                            p.B, p.H, E, g.dims.n_rel, chunks);
     trace_mark(p.stream, "drel_partial");
     const size_t per_chunk = (size_t)g.dims.n_rel * D;
-    drel_reduce_kernel<<<(unsigned)((per_chunk + 255) / 256), 256, 0, p.stream>>>(ws.part, p.d_rel, chunks, per_chunk, p.scale);
+    drel_reduce_kernel<<<(unsigned)((per_chunk + 255) / 256), 256, 0, p.stream>>>(ws.part, p.d_rel, chunks, per_chunk,
+                                                                                      (size_t)rel_anc(p.tree, 1) * D, p.scale);
     trace_mark(p.stream, "drel_reduce");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }

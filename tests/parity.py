@@ -24,6 +24,16 @@ def assert_close(name, got, want, tol):
     return rel
 
 
+def assert_max_norm(name, got, want, tol):
+    """||x-y||_inf / ||y||_inf <= tol."""
+    got = np.asarray(got, dtype=np.float64)
+    want = np.asarray(want, dtype=np.float64)
+    assert got.shape == want.shape and np.isfinite(got).all(), name
+    rel = np.abs(got - want).max() / np.abs(want).max()
+    assert rel <= tol, "%s: max-norm relative error %.3e > %.1e" % (name, rel, tol)
+    return rel
+
+
 def assert_small(name, got, ref_scale, tol):
     """For quantities that are exactly zero in theory (gradient of the ancestor relations)."""
     got = np.asarray(got, dtype=np.float64)

@@ -2,7 +2,7 @@
 import numpy as np
 import pytest
 
-from parity import TOL, assert_close, assert_small
+from parity import TOL, assert_close, assert_max_norm, assert_small
 
 pytestmark = pytest.mark.gpu
 
@@ -38,14 +38,21 @@ def run_case(n, k, flags, B, H, d, bf16, seed, std_qkv, backward=True, oracle_ba
         return
     dq, dk, dv, dr = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"])
     torch.cuda.synchronize()
-    rq, rk, rv, rr = ctwin.attn_bwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], scale, x["d_out"])
+    L, W = ref.L, k + 1
+    first_anc = 1 + 2 * L * W
+    # (1) against the exact gradient: max-norm relative error
+    exact = ctwin.attn_bwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], scale, x["d_out"])
+    for name, a, b in zip(("dq", "dk", "dv"), (dq, dk, dv), exact[:3]):
+        assert_max_norm(name, _np(a), b, tol)
+    assert_max_norm("d_rel", _np(dr)[:first_anc], exact[3][:first_anc], tol)
+    assert_small("d_rel[anc]", _np(dr)[first_anc:], np.abs(exact[3]).max(), tol)
+    # (2) against the oracle evaluating the row term d_out . out with the stored (rounded)
+    # forward output the library was given: element-wise as well
+    rq, rk, rv, rr = ctwin.attn_bwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], scale, x["d_out"], out=_np(out))
     assert_close("dq", _np(dq), rq, tol)
     assert_close("dk", _np(dk), rk, tol)
     assert_close("dv", _np(dv), rv, tol)
-    L, W = ref.L, k + 1
-    first_anc = 1 + 2 * L * W
     assert_close("d_rel", _np(dr)[:first_anc], rr[:first_anc], tol)
-    assert_small("d_rel[anc]", _np(dr)[first_anc:], np.abs(rr).max(), tol)
     # atomics-free, fixed order: a second run gives the same bits
     dq2, dk2, dv2, dr2 = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"])
     out2, lse2 = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale)

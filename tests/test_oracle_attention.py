@@ -157,3 +157,17 @@ def test_backward_structure():
     np.testing.assert_allclose(dq2[1], dq[0], rtol=1e-12)
     np.testing.assert_allclose(dk2[0], dk[0], rtol=1e-12)
     np.testing.assert_allclose(dv2[1], dv[0], rtol=1e-12)
+
+
+def test_backward_row_term_from_stored_output():
+    """sum_e P_e dP_e = d_out_u . out_u: passing the exact forward output reproduces the
+    exact gradient; passing a perturbed one changes dq, dk, d_rel but never dv."""
+    g, q, kk, v, r, go = _rand(16, 2, 0, B=2, H=2, d=4, seed=6)
+    out, _ = orc.attn_fwd(g, q, kk, v, r, 0.5)
+    exact = orc.attn_bwd(g, q, kk, v, r, 0.5, go)
+    same = orc.attn_bwd(g, q, kk, v, r, 0.5, go, out=out)
+    for a, b in zip(exact, same):
+        np.testing.assert_allclose(b, a, rtol=1e-11, atol=1e-13)
+    pert = orc.attn_bwd(g, q, kk, v, r, 0.5, go, out=out * 1.01)
+    np.testing.assert_allclose(pert[2], exact[2], rtol=1e-12, atol=1e-14)
+    assert np.abs(pert[0] - exact[0]).max() > 1e-6

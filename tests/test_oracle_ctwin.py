@@ -37,6 +37,9 @@ def test_attention(n, k, flags):
     cgrads = ctwin.attn_bwd(g, q, kk, v, r, 0.3, go)
     for a, b in zip(grads, cgrads):
         np.testing.assert_allclose(b, a, rtol=1e-11, atol=1e-12)
+    rounded = np.round(out * 64) / 64
+    for a, b in zip(orc.attn_bwd(g, q, kk, v, r, 0.3, go, out=rounded), ctwin.attn_bwd(g, q, kk, v, r, 0.3, go, out=rounded)):
+        np.testing.assert_allclose(b, a, rtol=1e-11, atol=1e-12)
     # batch slicing: entries outside [b0, b1) untouched, dr sums the slice only
     part = ctwin.attn_bwd(g, q, kk, v, r, 0.3, go, b0=1, b1=2)
     one = orc.attn_bwd(g, q[1:2], kk[1:2], v[1:2], r, 0.3, go[1:2])
