@@ -35,7 +35,8 @@ typedef enum {
     BPT_ERR_WORKSPACE = 3,    /* workspace missing or smaller than the size query says      */
     BPT_ERR_CUDA = 4,         /* a CUDA runtime call or launch failed                       */
     BPT_ERR_TIMEOUT = 5,      /* reserved: a bounded device-side wait expired               */
-    BPT_ERR_OVERFLOW = 6      /* edge count does not fit the 32-bit index arrays            */
+    BPT_ERR_OVERFLOW = 6,     /* edge count does not fit the 32-bit index arrays            */
+    BPT_ERR_SCRATCH_LIMIT = 7 /* problem needs more scratch than the built-in static array  */
 } bpt_status;
 
 /* flags of a graph */
@@ -140,6 +141,37 @@ bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt
                         const void* out, const float* lse, const void* d_out,
                         void* dq, void* dk, void* dv, float* d_rel,
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward pass for callers that must not allocate device memory (the paper has no
+ * counterpart; this is a deployment convenience).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plugin inside a host
+ * application that hands out tensors but no raw allocator, a real-time or safety-reviewed
+ * loop whose rules forbid allocation after start-up, a process whose memory pool already
+ * owns the whole device.  Such callers can provide the inputs and outputs of the
+ * backward, but have nowhere to get its workspace from.
+ *
+ * Same arguments, results and errors as bpt_attn_bwd, minus the workspace: the scratch
+ * is a 32 MiB array that lives inside the library's device image (every GPU that loads
+ * the library carries it until the process exits).  bpt_static_scratch_bytes() returns
+ * that limit; a problem whose bpt_attn_workspace_bytes(..., backward = 1) exceeds it is
+ * refused with BPT_ERR_SCRATCH_LIMIT before anything is launched (use bpt_attn_bwd with
+ * your own workspace then).  The call itself performs no cudaMalloc / cudaFree and calls
+ * no allocating library routine.
+ *
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call outside of any stream capture.  All calls on a device
+ * share the one array, and it keeps whatever the previous call left in it: the backward
+ * overwrites every part before reading it, so nothing needs clearing, but two calls whose
+ * GPU work overlaps (different streams, or different threads) would race on it -- keep
+ * them ordered on one stream.
+ */
+size_t bpt_static_scratch_bytes(void);
+bpt_status bpt_attn_bwd_static_scratch(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                       const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                       const void* out, const float* lse, const void* d_out,
+                                       void* dq, void* dk, void* dv, float* d_rel, void* cuda_stream);
 
 /*
  * Per-launch timing for benchmarks (no counterpart in the paper).  Between

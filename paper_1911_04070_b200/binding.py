@@ -18,7 +18,8 @@ BPT_BIDIR, BPT_LEFT_ONLY, BPT_MODE_PAD, BPT_MODE_ALG1 = 0, 1, 0, 2
 BPT_F32, BPT_BF16 = 0, 1
 
 EXPORTS = ("bpt_graph_dims_query", "bpt_build_graph", "bpt_attn_workspace_bytes", "bpt_attn_fwd",
-           "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end")
+           "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end",
+           "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch")
 
 
 class BptError(RuntimeError):
@@ -63,6 +64,11 @@ def load_library() -> ctypes.CDLL:
         lib.bpt_attn_bwd.restype = ctypes.c_int
         lib.bpt_attn_bwd.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
                                      vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.bpt_static_scratch_bytes.restype = sz
+        lib.bpt_static_scratch_bytes.argtypes = []
+        lib.bpt_attn_bwd_static_scratch.restype = ctypes.c_int
+        lib.bpt_attn_bwd_static_scratch.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp,
+                                                    f32, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.bpt_trace_begin.restype = ctypes.c_int
         lib.bpt_trace_begin.argtypes = [i32, vp]
         lib.bpt_trace_end.restype = ctypes.c_int
@@ -197,6 +203,26 @@ def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, work
                                 float(scale), _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq), _ptr(dk), _ptr(dv),
                                 _ptr(d_rel), _ptr(workspace), 0 if workspace is None else workspace.numel(),
                                 _stream()), "bpt_attn_bwd")
+    return dq, dk, dv, d_rel
+
+
+def bpt_static_scratch_bytes() -> int:
+    return int(load_library().bpt_static_scratch_bytes())
+
+
+def bpt_attn_bwd_static_scratch(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, dq, dk, dv, d_rel):
+    """Backward pass that takes its scratch from the library's built-in device array instead
+    of a workspace tensor, for callers that are not allowed to allocate device memory.  The
+    caller passes every input and output (this wrapper allocates nothing either); problems
+    above bpt_static_scratch_bytes() raise BptError with status 7.  Calls share the array:
+    keep them ordered on one stream."""
+    _check_layout(g, q, k, v, out, d_out, dq, dk, dv)
+    B, N, H, d = q.shape
+    with torch.cuda.device(q.device):
+        _check(load_library().bpt_attn_bwd_static_scratch(
+            ctypes.byref(g.c), B, H, d, _dtype_code(q), _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb), float(scale),
+            _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(d_rel), _stream()),
+            "bpt_attn_bwd_static_scratch")
     return dq, dk, dv, d_rel
 
 

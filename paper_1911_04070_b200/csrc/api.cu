@@ -118,6 +118,7 @@ extern "C" const char* bpt_status_str(bpt_status s) {
         case BPT_ERR_CUDA: return "CUDA error";
         case BPT_ERR_TIMEOUT: return "device-side wait timed out";
         case BPT_ERR_OVERFLOW: return "edge count exceeds 32-bit indices";
+        case BPT_ERR_SCRATCH_LIMIT: return "problem needs more scratch than the built-in static array holds";
     }
     return "unknown status";
 }
