@@ -165,7 +165,7 @@ def cpu_baseline(cfg):
 def run_ours(args, cfg_name, cfg):
     import torch
     import torch.distributed as dist
-    from paper_1911_04070_b200 import binding, synth
+    from paper_1911_04070_b200 import binding, shard, synth
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -200,8 +200,7 @@ def run_ours(args, cfg_name, cfg):
         if do_bwd:
             binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"], workspace=ws,
                                  dq=dq, dk=dk, dv=dv, d_rel=d_rel)
-            if world > 1:
-                dist.all_reduce(d_rel)
+            shard.allreduce_d_rel(d_rel)
 
     def barrier():
         if world > 1:
