@@ -14,15 +14,16 @@ template <typename T, int D, int U>
 __global__ void __launch_bounds__(256)
 fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col, const int32_t* __restrict__ rel,
                 const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
-                T* __restrict__ out, float* __restrict__ lse, int N, int H, int ngroups, float scale_log2e) {
+                T* __restrict__ out, float* __restrict__ lse, int N, int row0, int nrows, int H, int ngroups,
+                float scale_log2e) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
     const int nw = blockDim.x >> 5, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t bid = blockIdx.x;
-    const int u = N - 1 - (int)(bid % N);  // long span rows first
-    const int hg = (int)((bid / N) % ngroups);
-    const int b = (int)(bid / ((int64_t)N * ngroups));
+    const int u = row0 + nrows - 1 - (int)(bid % nrows);  // rows [row0, row0 + nrows), long span rows first
+    const int hg = (int)((bid / nrows) % ngroups);
+    const int b = (int)(bid / ((int64_t)nrows * ngroups));
     const int head = hg * M::HPW + lane / M::G;
     const bool head_ok = head < H;
     const int hc = head_ok ? head : H - 1;
@@ -121,28 +122,38 @@ int rows_kernel_warps(const bpt_graph& g) {
 }
 
 template <typename T, int D>
-static bpt_status launch_rows(const AttnProblem& p) {
+static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows) {
     using M = RowMap<T, D>;
     constexpr int U = 4;
     const bpt_graph& g = *p.g;
     const int N = g.dims.n_nodes;
     const int ngroups = (p.H + M::HPW - 1) / M::HPW;
     const int nw = rows_kernel_warps(g);
-    const int64_t blocks = (int64_t)p.B * N * ngroups;
+    const int64_t blocks = (int64_t)p.B * nrows * ngroups;
     if (blocks > 0x7fffffffll) return BPT_ERR_UNSUPPORTED;
     const size_t smem = nw > 1 ? (size_t)nw * 32 * (2 + M::EPL) * sizeof(float) : 0;
     fwd_rows_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (T*)p.out, p.lse, N, p.H, ngroups, p.scale * kLog2e);
+        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e);
     trace_mark(p.stream, "fwd_rows");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }
 
 size_t fwd_workspace_bytes(const bpt_graph&, int, int, int, bpt_dtype) { return 0; }
 
+bool fwd_tile_eligible(const AttnProblem& p);
+bpt_status launch_fwd_tile(const AttnProblem& p);
+
 bpt_status launch_fwd(const AttnProblem& p) {
-    if (p.dtype == BPT_F32) return p.d == 64 ? launch_rows<float, 64>(p) : launch_rows<float, 32>(p);
-    return p.d == 64 ? launch_rows<__nv_bfloat16, 64>(p) : launch_rows<__nv_bfloat16, 32>(p);
+    int row0 = 0, nrows = p.g->dims.n_nodes;
+    if (fwd_tile_eligible(p)) {  // token rows on the tensor cores, span rows below
+        const bpt_status s = launch_fwd_tile(p);
+        if (s != BPT_OK) return s;
+        row0 = p.tree.n;
+        nrows -= p.tree.n;
+    }
+    if (p.dtype == BPT_F32) return p.d == 64 ? launch_rows<float, 64>(p, row0, nrows) : launch_rows<float, 32>(p, row0, nrows);
+    return p.d == 64 ? launch_rows<__nv_bfloat16, 64>(p, row0, nrows) : launch_rows<__nv_bfloat16, 32>(p, row0, nrows);
 }
 
 }  // namespace bpt
