@@ -222,7 +222,7 @@ def run_ours(args, cfg_name, cfg):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    cap = min(args.steps * 8 + 8, 4000)
+    cap = min(args.steps * 16 + 8, 4000)
     binding.bpt_trace_begin(cap)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()

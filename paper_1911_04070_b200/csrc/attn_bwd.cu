@@ -42,7 +42,6 @@ static BwdWorkspace carve(const bpt_graph& g, int B, int H, int d, void* base) {
     return w;
 }
 
-size_t bwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype) { return carve(g, B, H, d, nullptr).bytes; }
 
 // ---------------------------------------------------------------------------------
 // A: by destination
@@ -53,15 +52,15 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
                const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
                const T* __restrict__ out, const float* __restrict__ lse, const T* __restrict__ d_out,
                T* __restrict__ dq, float* __restrict__ ws_p, float* __restrict__ ws_ds,
-               int N, int H, int ngroups, int64_t E, float scale) {
+               int N, int row0, int nrows, int H, int ngroups, int64_t e_first, int64_t E, float scale) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
     const int nw = blockDim.x >> 5, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t bid = blockIdx.x;
-    const int u = N - 1 - (int)(bid % N);
-    const int hg = (int)((bid / N) % ngroups);
-    const int b = (int)(bid / ((int64_t)N * ngroups));
+    const int u = row0 + nrows - 1 - (int)(bid % nrows);  // rows [row0, row0 + nrows), long span rows first
+    const int hg = (int)((bid / nrows) % ngroups);
+    const int b = (int)(bid / ((int64_t)nrows * ngroups));
     const int head = hg * M::HPW + lane / M::G;
     const bool head_ok = head < H;
     const int hc = head_ok ? head : H - 1;
@@ -114,7 +113,7 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
 #pragma unroll
                 for (int x = 0; x < EPL; ++x) acc[x] = fmaf(ds, kk[x], acc[x]);
                 if (sub == 0 && head_ok) {
-                    const size_t o = (eoff + (size_t)(e0 + j)) * H + head;
+                    const size_t o = (eoff + (size_t)(e0 + j - e_first)) * H + head;  // E edges kept per batch entry, from e_first on
                     ws_p[o] = p;
                     ws_ds[o] = ds;
                 }
@@ -366,7 +365,7 @@ static bpt_status launch_bwd_rows(const AttnProblem& p) {
     const size_t smem_a = nw > 1 ? (size_t)nw * 32 * M::EPL * sizeof(float) : 0;
     bwd_dst_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem_a, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, p.H, ngroups, E, p.scale);
+        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, 0, N, p.H, ngroups, 0, E, p.scale);
     trace_mark(p.stream, "bwd_dst");
 
     const size_t smem_b = nw > 1 ? (size_t)nw * 32 * (2 * M::EPL) * sizeof(float) : 0;
@@ -387,7 +386,17 @@ static bpt_status launch_bwd_rows(const AttnProblem& p) {
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }
 
+bool bwd_tile_eligible(const bpt_graph& g, int d, bpt_dtype dtype);
+size_t bwd_tile_workspace_bytes(const bpt_graph& g, int B, int H);
+bpt_status launch_bwd_tile(const AttnProblem& p);
+
+size_t bwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype) {
+    if (bwd_tile_eligible(g, d, dtype)) return bwd_tile_workspace_bytes(g, B, H);
+    return carve(g, B, H, d, nullptr).bytes;
+}
+
 bpt_status launch_bwd(const AttnProblem& p) {
+    if (bwd_tile_eligible(*p.g, p.d, p.dtype)) return launch_bwd_tile(p);
     if (p.dtype == BPT_F32) return p.d == 64 ? launch_bwd_rows<float, 64>(p) : launch_bwd_rows<float, 32>(p);
     return p.d == 64 ? launch_bwd_rows<__nv_bfloat16, 64>(p) : launch_bwd_rows<__nv_bfloat16, 32>(p);
 }

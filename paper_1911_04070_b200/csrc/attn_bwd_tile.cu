@@ -1,0 +1,581 @@
+// Tiled backward for the token rows (arXiv 1911.04070: gradient of the Sec. 3.4 equation over
+// the contextual edges of Sec. 3.2.2), bf16, head size 64.
+//
+// One CTA = 64 consecutive tokens of one (batch entry, head), 4 warps.  As in the tiled forward
+// the nodes a token attends at one (side, level) are one contiguous range, so per chunk the CTA
+// stages the union range of K and V rows once.  The token's self loop is folded into the
+// level-0 left chunk: node i follows its left neighbours directly, and the relation ids
+// self = 0, left(0, o) = 1 + o are consecutive, so the self loop is simply offset 0 of a range
+// that ends at the token itself.
+//
+//   phase 1 (a warp owns 16 query rows):  S = Q K^T + skewed Q R^T,  P = exp(S - lse),
+//            dP = dO V^T,  dS = P (dP - dO.O);  dQ += dS K + skew(dS) R;
+//            P, dS and the skewed dS (indexed by relation offset) go to shared memory as bf16
+//   phase 2 (a warp owns 16 staged key rows):  dK_part = dS^T Q,  dV_part = P^T dO for the
+//            chunk's node range and dR_part = skew(dS)^T Q, written to the workspace.
+//
+// Nothing is accumulated across CTAs here: bwd_gather_kernel sums, for every source node, the
+// partial rows of the tiles whose range covers it, in tile order (no atomics, fixed order), and
+// drel_sum kernels do the same for the relation table.
+#include "bpt_internal.cuh"
+#include "mma_tools.cuh"
+#include "row_map.cuh"
+#include "tile_geom.cuh"
+
+namespace bpt {
+
+size_t bwd_span_ext_floats(const TreeParams& t, int n_pairs);
+size_t bwd_span_slab_floats(const TreeParams& t, int n_pairs);
+bpt_status launch_bwd_span(const AttnProblem& p, int pair0, int n_pairs, float* ext_dq, float* aff_slab);
+
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kKvRows = 208;      // staged K / V rows per chunk
+constexpr int kRelRows = 80;      // staged relation rows per chunk (k + 2 <= 66, padded to 16)
+constexpr int kQrStride = 76;     // floats per row of the per-warp Q R^T scratch
+constexpr int kPStride = 432;     // bytes per token row of the P / dS tiles (208 bf16 + 16: odd number of 16-byte chunks)
+constexpr int kSkewStride = 176;  // bytes per token row of the skewed dS tile (80 bf16 + 16)
+constexpr int kMaxChunks = 2 * kMaxLevels;
+constexpr int kDrelGroups = 32;   // first stage of the d_rel sum
+
+struct ChunkPlan {
+    int n_left, n_right;
+    int slab_row0[kMaxChunks + 1];  // first reserved partial row of each chunk; [chunks] = rows per tile
+    int rel_rows;                   // relation rows reserved per chunk in the d_rel partials (multiple of 16)
+};
+
+struct BwdTileSmem {
+    static constexpr int q_bytes = kTileTokens * 128;
+    static constexpr int kv_bytes = kKvRows * 128;
+    static constexpr int r_bytes = kRelRows * 128;
+    static constexpr int qr_bytes = 4 * 16 * kQrStride * 4;
+    static constexpr int p_bytes = kTileTokens * kPStride;
+    static constexpr int skew_bytes = kTileTokens * kSkewStride;
+    static constexpr int row_bytes = 2 * kTileTokens * 4;  // lse, delta
+    static constexpr int fixed = 2 * q_bytes + 2 * kv_bytes + r_bytes + qr_bytes + 2 * p_bytes + skew_bytes + row_bytes;
+    static size_t bytes(int chunks) { return (size_t)fixed + (size_t)chunks * (kTileTokens * 8 + 8); }
+};
+
+__global__ void __launch_bounds__(128)
+bwd_tile_kernel(TreeParams t, ChunkPlan plan,
+                const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+                const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
+                const __nv_bfloat16* __restrict__ out, const float* __restrict__ lse,
+                const __nv_bfloat16* __restrict__ d_out, __nv_bfloat16* __restrict__ dq,
+                int2* __restrict__ tile_range, float* __restrict__ slabs, float* __restrict__ drel_part,
+                int H, int pair0, float scale) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* q_s = smem;
+    unsigned char* g_s = q_s + BwdTileSmem::q_bytes;   // d_out tile
+    unsigned char* k_s = g_s + BwdTileSmem::q_bytes;
+    unsigned char* v_s = k_s + BwdTileSmem::kv_bytes;
+    unsigned char* r_s = v_s + BwdTileSmem::kv_bytes;
+    float* qr_s = reinterpret_cast<float*>(r_s + BwdTileSmem::r_bytes);
+    unsigned char* p_s = reinterpret_cast<unsigned char*>(qr_s) + BwdTileSmem::qr_bytes;
+    unsigned char* ds_s = p_s + BwdTileSmem::p_bytes;
+    unsigned char* sk_s = ds_s + BwdTileSmem::p_bytes;
+    float* lse_s = reinterpret_cast<float*>(sk_s + BwdTileSmem::skew_bytes);
+    float* delta_s = lse_s + kTileTokens;
+    int2* bnd = reinterpret_cast<int2*>(delta_s + kTileTokens);
+    const int n_left = plan.n_left, n_right = plan.n_right, chunks = n_left + n_right;
+    int2* crange = bnd + chunks * kTileTokens;
+
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int g = lane >> 2, c2 = (lane & 3) * 2;
+    const int tile = blockIdx.x, tiles = gridDim.x, t0 = tile * kTileTokens;
+    const int pair = pair0 + blockIdx.y, b = pair / H, h = pair % H;
+    const int N = 2 * t.n - 1;
+    const size_t rs = (size_t)H * 64;
+    const size_t boff = (size_t)b * N * rs + (size_t)h * 64;
+    const uint32_t q_u = smem_u32(q_s), g_u = smem_u32(g_s), k_u = smem_u32(k_s), v_u = smem_u32(v_s),
+                   r_u = smem_u32(r_s), p_u = smem_u32(p_s), ds_u = smem_u32(ds_s), sk_u = smem_u32(sk_s);
+    const float scale_log2e = scale * kLog2e;
+
+    // ---- prologue: Q and dO tiles, out tile (into the K buffer) for the row term, row ranges ----
+    for (int idx = tid; idx < kTileTokens * 8; idx += 128) {
+        const int row = idx >> 3, ch = idx & 7;
+        const size_t src = boff + (size_t)(t0 + row) * rs + ch * 8;
+        cp_async16(q_u + tile_off(row, ch), q + src);
+        cp_async16(g_u + tile_off(row, ch), d_out + src);
+        cp_async16(k_u + tile_off(row, ch), out + src);
+    }
+    cp_async_commit();
+    if (tid < kTileTokens) {
+        fill_row_bounds(t, t0, tid, n_left, n_right, bnd);
+        // the self loop joins the level-0 left range: it ends at the token itself
+        const int i = t0 + tid;
+        const int2 v0 = bnd[tid];
+        bnd[tid] = v0.x > v0.y ? make_int2(i, i) : make_int2(v0.x, i);
+        lse_s[tid] = lse[((size_t)b * N + i) * H + h] * kLog2e;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    {   // delta_i = d_out_i . out_i: two threads per row
+        const int row = tid >> 1, half = tid & 1;
+        float acc = 0.f;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            const uint4 a = *reinterpret_cast<const uint4*>(g_s + tile_off(row, half * 4 + ch));
+            const uint4 o = *reinterpret_cast<const uint4*>(k_s + tile_off(row, half * 4 + ch));
+            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, ow[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                acc = fmaf(__uint_as_float(aw[x] << 16), __uint_as_float(ow[x] << 16), acc);
+                acc = fmaf(__uint_as_float(aw[x] & 0xffff0000u), __uint_as_float(ow[x] & 0xffff0000u), acc);
+            }
+        }
+        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+        if (half == 0) delta_s[row] = acc;
+    }
+    for (int c = w; c < chunks; c += 4) {
+        const int2 a = rows_union(bnd + c * kTileTokens, 0, 32, lane);
+        const int2 bb = rows_union(bnd + c * kTileTokens, 32, 32, lane);
+        if (lane == 0) {
+            const int2 u = make_int2(min(a.x, bb.x), max(a.y, bb.y));
+            crange[c] = u;
+            if (blockIdx.y == 0 && pair0 == 0) {
+                // empty ranges keep the table monotone over the tiles: left levels are missing for a
+                // prefix of the tiles, right levels for a suffix
+                const int n_l = t.n >> (c >= n_left ? c - n_left : c);
+                tile_range[(size_t)c * tiles + tile] = u.x <= u.y ? u : (c >= n_left ? make_int2(n_l, n_l - 1) : make_int2(0, -1));
+            }
+        }
+    }
+
+    const int r0 = w * 16;
+    uint32_t qa[4][4], ga[4][4];
+    load_a_frags(q_u, r0, lane, qa);
+    load_a_frags(g_u, r0, lane, ga);
+    float acc_q[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) { acc_q[nt][0] = acc_q[nt][1] = acc_q[nt][2] = acc_q[nt][3] = 0.f; }
+
+    float* qr_w = qr_s + w * 16 * kQrStride;
+    const int W = t.k + 1;
+    float* slab_cta = slabs + ((size_t)blockIdx.y * tiles + tile) * plan.slab_row0[chunks] * 128;
+    float* drel_cta = drel_part + ((size_t)blockIdx.y * tiles + tile) * chunks * plan.rel_rows * 64;
+
+    for (int c = 0; c < chunks; ++c) {
+        __syncthreads();  // previous chunk's tiles are free (and, first time, delta / crange are visible)
+        const int2 cr = crange[c];
+        if (cr.x > cr.y) {  // no token of the tile reaches this level: its d_rel partial is zero
+            float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)c * plan.rel_rows * 64);
+            for (int idx = tid; idx < plan.rel_rows * 16; idx += 128) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+            continue;
+        }
+        const int side = c >= n_left;
+        const int level = side ? c - n_left : c;
+        const int n_l = t.n >> level;
+        const int id_base = node_id(t.n, level, 0);
+        const int rel_base = c == 0 ? 0 : (side ? rel_right(t, level, 0) : rel_left(t, level, 0));
+        const int n_rel_c = c == 0 ? W + 1 : W;
+        const int base = cr.x & ~15;
+        const int kend = cr.y - base;
+        const int nr = min(kKvRows, (kend + 1 + 31 + 15) & ~15);
+
+        for (int idx = tid; idx < nr * 8; idx += 128) {
+            const int row = idx >> 3, ch = idx & 7;
+            const int node = min(base + row, n_l - 1);
+            const size_t src = boff + (size_t)(id_base + node) * rs + ch * 8;
+            cp_async16(k_u + tile_off(row, ch), k + src);
+            cp_async16(v_u + tile_off(row, ch), v + src);
+        }
+        for (int idx = tid; idx < kRelRows * 8; idx += 128) {
+            const int row = idx >> 3, ch = idx & 7;
+            if (row < n_rel_c) cp_async16(r_u + tile_off(row, ch), r + (size_t)(rel_base + row) * 64 + ch * 8);
+            else *reinterpret_cast<uint4*>(r_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
+        }
+        cp_async_commit();
+        for (int idx = tid; idx < kTileTokens * (kSkewStride / 16); idx += 128)
+            *reinterpret_cast<uint4*>(sk_s + idx * 16) = make_uint4(0, 0, 0, 0);
+        cp_async_wait<0>();
+        __syncthreads();
+
+        // ================= phase 1: this warp's 16 query rows =================
+        const int2* bc = bnd + c * kTileTokens;
+        const int2 wr = rows_union(bc, r0, 16, lane);
+        const bool w_any = wr.x <= wr.y;
+        if (w_any) {  // Q R^T for the chunk's relation rows -> per-warp scratch
+#pragma unroll
+            for (int np = 0; np < kRelRows / 16; ++np) {
+                if (np * 16 < n_rel_c) {
+                    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks) {
+                        uint32_t bf[4];
+                        load_b_rows(r_u, np * 16, ks, lane, bf);
+                        mma_bf16(acc[0], qa[ks], bf[0], bf[1]);
+                        mma_bf16(acc[1], qa[ks], bf[2], bf[3]);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const int col = np * 16 + j * 8 + c2;
+                        if (col < kQrStride) {
+                            *reinterpret_cast<float2*>(qr_w + g * kQrStride + col) = make_float2(acc[j][0], acc[j][1]);
+                            *reinterpret_cast<float2*>(qr_w + (g + 8) * kQrStride + col) = make_float2(acc[j][2], acc[j][3]);
+                        }
+                    }
+                }
+            }
+        }
+        __syncwarp();
+
+        const int2 ba = bc[r0 + g], bb = bc[r0 + g + 8];
+        const int lo_r[2] = {ba.x, bb.x}, hi_r[2] = {ba.y, bb.y};
+        const float lse_r[2] = {lse_s[r0 + g], lse_s[r0 + g + 8]};
+        const float del_r[2] = {delta_s[r0 + g], delta_s[r0 + g + 8]};
+        const int w_lo = w_any ? wr.x - base : 1 << 30, w_hi = w_any ? wr.y - base : -1;
+        for (int kb = 0; kb <= kend; kb += 32) {
+            unsigned char* p_row0 = p_s + (r0 + g) * kPStride + (kb + c2) * 2;
+            unsigned char* d_row0 = ds_s + (r0 + g) * kPStride + (kb + c2) * 2;
+            if (kb + 31 < w_lo || kb > w_hi) {  // nothing of this warp's rows here: zeros for phase 2
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    *reinterpret_cast<uint32_t*>(p_row0 + j * 16) = 0u;
+                    *reinterpret_cast<uint32_t*>(p_row0 + 8 * kPStride + j * 16) = 0u;
+                    *reinterpret_cast<uint32_t*>(d_row0 + j * 16) = 0u;
+                    *reinterpret_cast<uint32_t*>(d_row0 + 8 * kPStride + j * 16) = 0u;
+                }
+                continue;
+            }
+            float s[4][4], dp[4][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
+                dp[j][0] = dp[j][1] = dp[j][2] = dp[j][3] = 0.f;
+            }
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+                for (int np = 0; np < 2; ++np) {
+                    uint32_t bf[4];
+                    load_b_rows(k_u, kb + np * 16, ks, lane, bf);
+                    mma_bf16(s[np * 2], qa[ks], bf[0], bf[1]);
+                    mma_bf16(s[np * 2 + 1], qa[ks], bf[2], bf[3]);
+                    load_b_rows(v_u, kb + np * 16, ks, lane, bf);
+                    mma_bf16(dp[np * 2], ga[ks], bf[0], bf[1]);
+                    mma_bf16(dp[np * 2 + 1], ga[ks], bf[2], bf[3]);
+                }
+            }
+            uint32_t da[2][4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float pv[4], dv[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int hh = e >> 1;
+                    const int m = base + kb + j * 8 + c2 + (e & 1);
+                    const bool ok = m >= lo_r[hh] && m <= hi_r[hh];
+                    float p = 0.f, d = 0.f;
+                    if (ok) {
+                        const int off = side ? m - lo_r[hh] : hi_r[hh] - m;
+                        const float bias = qr_w[(g + hh * 8) * kQrStride + off];
+                        p = fast_exp2(fmaf(s[j][e] + bias, scale_log2e, -lse_r[hh]));
+                        d = p * (dp[j][e] - del_r[hh]);
+                        *reinterpret_cast<__nv_bfloat16*>(sk_s + (r0 + g + hh * 8) * kSkewStride + off * 2) = __float2bfloat16_rn(d);
+                    }
+                    pv[e] = p; dv[e] = d;
+                }
+                const uint32_t p01 = pack_bf16(pv[0], pv[1]), p23 = pack_bf16(pv[2], pv[3]);
+                const uint32_t d01 = pack_bf16(dv[0], dv[1]), d23 = pack_bf16(dv[2], dv[3]);
+                *reinterpret_cast<uint32_t*>(p_row0 + j * 16) = p01;
+                *reinterpret_cast<uint32_t*>(p_row0 + 8 * kPStride + j * 16) = p23;
+                *reinterpret_cast<uint32_t*>(d_row0 + j * 16) = d01;
+                *reinterpret_cast<uint32_t*>(d_row0 + 8 * kPStride + j * 16) = d23;
+                da[j >> 1][(j & 1) * 2] = d01;
+                da[j >> 1][(j & 1) * 2 + 1] = d23;
+            }
+            // dQ += dS K
+#pragma unroll
+            for (int kk = 0; kk < 2; ++kk) {
+#pragma unroll
+                for (int np = 0; np < 4; ++np) {
+                    uint32_t bf[4];
+                    load_b_cols(k_u, kb + kk * 16, np, lane, bf);
+                    mma_bf16(acc_q[np * 2], da[kk], bf[0], bf[1]);
+                    mma_bf16(acc_q[np * 2 + 1], da[kk], bf[2], bf[3]);
+                }
+            }
+        }
+        __syncwarp();
+        if (w_any) {  // dQ += skew(dS) R_chunk (this warp wrote its own 16 rows of the skew tile)
+#pragma unroll
+            for (int kk = 0; kk < kRelRows / 16; ++kk) {
+                if (kk * 16 < n_rel_c) {
+                    uint32_t a[4];
+                    load_a_plain(sk_u, kSkewStride, r0, kk * 16, lane, a);
+#pragma unroll
+                    for (int np = 0; np < 4; ++np) {
+                        uint32_t bf[4];
+                        load_b_cols(r_u, kk * 16, np, lane, bf);
+                        mma_bf16(acc_q[np * 2], a, bf[0], bf[1]);
+                        mma_bf16(acc_q[np * 2 + 1], a, bf[2], bf[3]);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+
+        // ================= phase 2: this warp's key rows and relation offsets =================
+        const int n_jt = (kend >> 4) + 1;
+        for (int jt = w; jt < n_jt; jt += 4) {
+            float ak[8][4], av[8][4];
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                ak[nt][0] = ak[nt][1] = ak[nt][2] = ak[nt][3] = 0.f;
+                av[nt][0] = av[nt][1] = av[nt][2] = av[nt][3] = 0.f;
+            }
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t a_ds[4], a_p[4];
+                load_a_trans(ds_u, kPStride, ks * 16, jt * 16, lane, a_ds);
+                load_a_trans(p_u, kPStride, ks * 16, jt * 16, lane, a_p);
+#pragma unroll
+                for (int np = 0; np < 4; ++np) {
+                    uint32_t bf[4];
+                    load_b_cols(q_u, ks * 16, np, lane, bf);
+                    mma_bf16(ak[np * 2], a_ds, bf[0], bf[1]);
+                    mma_bf16(ak[np * 2 + 1], a_ds, bf[2], bf[3]);
+                    load_b_cols(g_u, ks * 16, np, lane, bf);
+                    mma_bf16(av[np * 2], a_p, bf[0], bf[1]);
+                    mma_bf16(av[np * 2 + 1], a_p, bf[2], bf[3]);
+                }
+            }
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int m = base + jt * 16 + g + hh * 8;
+                if (m >= cr.x && m <= cr.y) {
+                    float* dst = slab_cta + (size_t)(plan.slab_row0[c] + m - cr.x) * 128 + c2;
+#pragma unroll
+                    for (int nt = 0; nt < 8; ++nt) {
+                        *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ak[nt][hh * 2], ak[nt][hh * 2 + 1]);
+                        *reinterpret_cast<float2*>(dst + 64 + nt * 8) = make_float2(av[nt][hh * 2], av[nt][hh * 2 + 1]);
+                    }
+                }
+            }
+        }
+        const int n_ot = plan.rel_rows >> 4;
+        for (int ot = 3 - w; ot < n_ot; ot += 4) {  // warps in reverse order: warp 3 has the fewest key tiles
+            float ar[8][4];
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) { ar[nt][0] = ar[nt][1] = ar[nt][2] = ar[nt][3] = 0.f; }
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                uint32_t a[4];
+                load_a_trans(sk_u, kSkewStride, ks * 16, ot * 16, lane, a);
+#pragma unroll
+                for (int np = 0; np < 4; ++np) {
+                    uint32_t bf[4];
+                    load_b_cols(q_u, ks * 16, np, lane, bf);
+                    mma_bf16(ar[np * 2], a, bf[0], bf[1]);
+                    mma_bf16(ar[np * 2 + 1], a, bf[2], bf[3]);
+                }
+            }
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const int o = ot * 16 + g + hh * 8;
+                float* dst = drel_cta + ((size_t)c * plan.rel_rows + o) * 64 + c2;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt)
+                    *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ar[nt][hh * 2], ar[nt][hh * 2 + 1]);
+            }
+        }
+    }
+
+    // ---- epilogue: dq = scale * acc, rounded once to bf16, coalesced stores through the Q tile ----
+    __syncthreads();
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g, nt) + c2 * 2) = pack_bf16(acc_q[nt][0] * scale, acc_q[nt][1] * scale);
+        *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g + 8, nt) + c2 * 2) = pack_bf16(acc_q[nt][2] * scale, acc_q[nt][3] * scale);
+    }
+    __syncwarp();
+    for (int idx = lane; idx < 16 * 8; idx += 32) {
+        const int row = r0 + (idx >> 3), ch = idx & 7;
+        *reinterpret_cast<uint4*>(dq + boff + (size_t)(t0 + row) * rs + ch * 8) =
+            *reinterpret_cast<const uint4*>(q_s + tile_off(row, ch));
+    }
+}
+
+// dk, dv of every node: the partial rows of the tiles whose chunk range covers the node (both
+// sides), in tile order, plus for a token the row the span pass left for it (the affiliated
+// edges into its L ancestors).  One warp per (pair, node); lanes 0..15 hold four channels of dk
+// each, lanes 16..31 four channels of dv.
+__global__ void __launch_bounds__(256)
+bwd_gather_kernel(TreeParams t, ChunkPlan plan, const int2* __restrict__ tile_range, const float* __restrict__ slabs,
+                  const float* __restrict__ aff_slab,
+                  __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+                  int H, int pair0, int n_pairs, int tiles, float scale) {
+    const int lane = threadIdx.x & 31;
+    const int N = 2 * t.n - 1;
+    const int64_t wid = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (wid >= (int64_t)n_pairs * N) return;
+    const int pl = (int)(wid / N);              // pair inside this pass
+    const int vtx = N - 1 - (int)(wid % N);     // coarse nodes (many tiles each) first
+    const int pair = pair0 + pl, b = pair / H, h = pair % H;
+    const int l = node_level(t.n, vtx), m = vtx - node_id(t.n, l, 0);
+    const int chunks = plan.n_left + plan.n_right;
+    const size_t tile_rows = (size_t)plan.slab_row0[chunks];
+    const float* slab_pair = slabs + (size_t)pl * tiles * tile_rows * 128;
+
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int side = 0; side < 2; ++side) {
+        if (l >= (side ? plan.n_right : plan.n_left)) continue;
+        const int c = side ? plan.n_left + l : l;
+        const int2* tr = tile_range + (size_t)c * tiles;
+        int lo = 0, hi = tiles;  // first tile whose range ends at or beyond m
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (tr[mid].y >= m) hi = mid; else lo = mid + 1; }
+        const int ta = lo;
+        hi = tiles;              // first tile whose range starts beyond m
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (tr[mid].x > m) hi = mid; else lo = mid + 1; }
+        const int tb = lo;
+        for (int T = ta; T < tb; ++T) {
+            const int row = plan.slab_row0[c] + m - tr[T].x;
+            const float4 x = __ldg(reinterpret_cast<const float4*>(slab_pair + ((size_t)T * tile_rows + row) * 128) + lane);
+            acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+        }
+    }
+    const size_t rs = (size_t)H * 64;
+    const size_t boff = (size_t)b * N * rs + (size_t)h * 64;
+    const int ch4 = (lane & 15) * 4;
+    if (l == 0) {
+        const float4 x = __ldg(reinterpret_cast<const float4*>(aff_slab + ((size_t)pl * t.n + m) * 128) + lane);
+        acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+    }
+    const float f = lane < 16 ? scale : 1.f;
+    __nv_bfloat16* dst = (lane < 16 ? dk : dv) + boff + (size_t)vtx * rs + ch4;
+    *reinterpret_cast<uint2*>(dst) = make_uint2(pack_bf16(acc.x * f, acc.y * f), pack_bf16(acc.z * f, acc.w * f));
+}
+
+// d_rel, first stage: the CTAs of one pass in kDrelGroups groups, each summed in CTA order.
+// x indexes (chunk, offset, channel) of the per-CTA partial tables.
+__global__ void drel_group_kernel(const float* __restrict__ part, float* __restrict__ grp, int n_ctas, size_t per_cta) {
+    const size_t x = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= per_cta) return;
+    const int gi = blockIdx.y;
+    const int per = (n_ctas + kDrelGroups - 1) / kDrelGroups;
+    const int c0 = min(gi * per, n_ctas), c1 = min(c0 + per, n_ctas);
+    float acc = 0.f;
+    for (int c = c0; c < c1; ++c) acc += part[(size_t)c * per_cta + x];
+    grp[(size_t)gi * per_cta + x] = acc;
+}
+
+// d_rel, second stage: one thread per (relation row, channel).  Rows that no chunk covers (and
+// the ancestor rows) are zero.  With `accumulate` the pass adds to what earlier passes wrote.
+__global__ void drel_final_kernel(TreeParams t, ChunkPlan plan, const float* __restrict__ grp, float* __restrict__ d_rel,
+                                  int n_rel, size_t per_cta, float scale, int accumulate) {
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= n_rel * 64) return;
+    const int rid = x >> 6, ch = x & 63;
+    const int W = t.k + 1;
+    int c = -1, off = 0;
+    if (rid <= W) { c = 0; off = rid; }               // self and left level 0 live in chunk 0
+    else if (rid < 1 + t.L * W) { const int j = (rid - 1) / W; if (j < plan.n_left) { c = j; off = (rid - 1) % W; } }
+    else if (rid < 1 + 2 * t.L * W) { const int j = (rid - 1 - t.L * W) / W; if (j < plan.n_right) { c = plan.n_left + j; off = (rid - 1 - t.L * W) % W; } }
+    float acc = 0.f;
+    if (c >= 0) {
+        const size_t at = ((size_t)c * plan.rel_rows + off) * 64 + ch;
+        for (int gi = 0; gi < kDrelGroups; ++gi) acc += grp[(size_t)gi * per_cta + at];
+    }
+    d_rel[x] = accumulate ? d_rel[x] + acc * scale : acc * scale;
+}
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct TileWorkspace {
+    int2* tile_range;
+    float *aff_slab, *ext_dq, *slabs, *drel_part, *drel_grp;
+    int pairs_per_pass;
+    size_t bytes;
+};
+
+constexpr size_t kPassBytes = (size_t)3 << 30;  // partial rows kept per pass
+
+ChunkPlan make_plan(const TreeParams& t) {
+    ChunkPlan p{};
+    context_levels(t, &p.n_left, &p.n_right);
+    int at = 0;
+    for (int c = 0; c < p.n_left + p.n_right; ++c) {
+        const int level = c >= p.n_left ? c - p.n_left : c;
+        p.slab_row0[c] = at;
+        at += (kTileTokens >> level) + t.kc + 3;  // upper bound of a tile's union range at this level
+    }
+    p.slab_row0[p.n_left + p.n_right] = at;
+    p.rel_rows = (t.k + 2 + 15) & ~15;
+    return p;
+}
+
+TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, int B, int H, void* base) {
+    const int chunks = plan.n_left + plan.n_right, tiles = t.n / kTileTokens;
+    const size_t per_pair = ((size_t)tiles * ((size_t)plan.slab_row0[chunks] * 128 + (size_t)chunks * plan.rel_rows * 64) +
+                             bwd_span_slab_floats(t, 1) + bwd_span_ext_floats(t, 1)) * sizeof(float);
+    TileWorkspace w;
+    size_t pairs = kPassBytes / per_pair;
+    if (pairs < 1) pairs = 1;
+    if (pairs > (size_t)B * H) pairs = (size_t)B * H;
+    w.pairs_per_pass = (int)pairs;
+    char* c = (char*)base;
+    size_t off = 0;
+    w.tile_range = (int2*)(c + off); off += align256(sizeof(int2) * chunks * tiles);
+    w.aff_slab = (float*)(c + off); off += align256(sizeof(float) * bwd_span_slab_floats(t, (int)pairs));
+    w.ext_dq = (float*)(c + off); off += align256(sizeof(float) * bwd_span_ext_floats(t, (int)pairs));
+    w.slabs = (float*)(c + off); off += align256(sizeof(float) * pairs * tiles * plan.slab_row0[chunks] * 128);
+    w.drel_part = (float*)(c + off); off += align256(sizeof(float) * pairs * tiles * chunks * plan.rel_rows * 64);
+    w.drel_grp = (float*)(c + off); off += align256(sizeof(float) * kDrelGroups * chunks * plan.rel_rows * 64);
+    w.bytes = off;
+    return w;
+}
+
+}  // namespace
+
+bool bwd_tile_eligible(const bpt_graph& g, int d, bpt_dtype dtype) {
+    return tile_path(g.dims.n, g.dims.k, d, dtype == BPT_BF16);
+}
+
+size_t bwd_tile_workspace_bytes(const bpt_graph& g, int B, int H) {
+    TreeParams t;
+    tree_params_from_dims(g.dims, &t);
+    return carve_tile(t, make_plan(t), B, H, nullptr).bytes;
+}
+
+
+bpt_status launch_bwd_tile(const AttnProblem& p) {
+    const TreeParams& t = p.tree;
+    const ChunkPlan plan = make_plan(t);
+    const int chunks = plan.n_left + plan.n_right, tiles = t.n / kTileTokens, N = 2 * t.n - 1;
+    const TileWorkspace ws = carve_tile(t, plan, p.B, p.H, p.workspace);
+    const size_t smem = BwdTileSmem::bytes(chunks);
+    if (smem > 227 * 1024) return BPT_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(bwd_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return BPT_ERR_CUDA;
+
+    const int total = p.B * p.H;
+    const size_t per_cta = (size_t)chunks * plan.rel_rows * 64;
+    for (int pair0 = 0; pair0 < total; pair0 += ws.pairs_per_pass) {
+        const int np = min(ws.pairs_per_pass, total - pair0);
+        if (np > 65535) return BPT_ERR_UNSUPPORTED;
+        // span rows: dq of the spans and, per token, the affiliated edges' share of dk / dv
+        const bpt_status s = launch_bwd_span(p, pair0, np, ws.ext_dq, ws.aff_slab);
+        if (s != BPT_OK) return s;
+        bwd_tile_kernel<<<dim3(tiles, np), 128, smem, p.stream>>>(
+            t, plan, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
+            (const __nv_bfloat16*)p.rel_emb, (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out,
+            (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale);
+        trace_mark(p.stream, "bwd_tile");
+        const int64_t warps = (int64_t)np * N;
+        bwd_gather_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, p.stream>>>(
+            t, plan, ws.tile_range, ws.slabs, ws.aff_slab, (__nv_bfloat16*)p.dk, (__nv_bfloat16*)p.dv,
+            p.H, pair0, np, tiles, p.scale);
+        trace_mark(p.stream, "bwd_gather");
+        drel_group_kernel<<<dim3((unsigned)((per_cta + 255) / 256), kDrelGroups), 256, 0, p.stream>>>(
+            ws.drel_part, ws.drel_grp, np * tiles, per_cta);
+        trace_mark(p.stream, "drel_group");
+        drel_final_kernel<<<(p.g->dims.n_rel * 64 + 255) / 256, 256, 0, p.stream>>>(
+            t, plan, ws.drel_grp, p.d_rel, p.g->dims.n_rel, per_cta, p.scale, pair0 > 0);
+        trace_mark(p.stream, "drel_final");
+    }
+    return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
+}
+
+}  // namespace bpt

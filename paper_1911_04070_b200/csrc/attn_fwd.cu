@@ -4,6 +4,7 @@
 // registers, and the per-warp states are merged in a fixed order through shared memory.
 #include "bpt_internal.cuh"
 #include "row_map.cuh"
+#include "tile_geom.cuh"
 
 namespace bpt {
 
@@ -139,19 +140,23 @@ static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows) {
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }
 
-size_t fwd_workspace_bytes(const bpt_graph&, int, int, int, bpt_dtype) { return 0; }
-
-bool fwd_tile_eligible(const AttnProblem& p);
 bpt_status launch_fwd_tile(const AttnProblem& p);
+size_t fwd_span_workspace_bytes(const TreeParams& t, int B, int H);
+bpt_status launch_fwd_span(const AttnProblem& p);
+
+size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype) {
+    if (!tile_path(g.dims.n, g.dims.k, d, dtype == BPT_BF16)) return 0;
+    TreeParams t;
+    tree_params_from_dims(g.dims, &t);
+    return fwd_span_workspace_bytes(t, B, H);
+}
 
 bpt_status launch_fwd(const AttnProblem& p) {
-    int row0 = 0, nrows = p.g->dims.n_nodes;
-    if (fwd_tile_eligible(p)) {  // token rows on the tensor cores, span rows below
+    if (tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16)) {  // token rows and span rows on the tensor cores
         const bpt_status s = launch_fwd_tile(p);
-        if (s != BPT_OK) return s;
-        row0 = p.tree.n;
-        nrows -= p.tree.n;
+        return s != BPT_OK ? s : launch_fwd_span(p);
     }
+    const int row0 = 0, nrows = p.g->dims.n_nodes;
     if (p.dtype == BPT_F32) return p.d == 64 ? launch_rows<float, 64>(p, row0, nrows) : launch_rows<float, 32>(p, row0, nrows);
     return p.d == 64 ? launch_rows<__nv_bfloat16, 64>(p, row0, nrows) : launch_rows<__nv_bfloat16, 32>(p, row0, nrows);
 }

@@ -23,7 +23,6 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kKvRows = 208;     // staged K / V rows per chunk (union range + alignment slack)
 constexpr int kRelRows = 80;     // staged relation rows per chunk (k + 1 <= 72, padded to 16)
 constexpr int kQrStride = 76;    // floats per row of the per-warp Q R^T scratch
-constexpr int kMaxK = 64;        // largest k this kernel takes
 
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -276,10 +275,6 @@ fwd_tile_kernel(TreeParams t, int n_left, int n_right,
 }
 
 }  // namespace
-
-bool fwd_tile_eligible(const AttnProblem& p) {
-    return p.dtype == BPT_BF16 && p.d == 64 && p.tree.n >= kTileTokens && p.tree.k <= kMaxK;
-}
 
 // Token rows of the forward on the tensor cores; the span rows are left to the caller.
 bpt_status launch_fwd_tile(const AttnProblem& p) {

@@ -69,4 +69,19 @@ __device__ __forceinline__ void load_b_cols(uint32_t tile_base, int row0, int np
     ldsm_x4_t(tile_base + tile_off(r, np * 2 + cj), b[0], b[1], b[2], b[3]);
 }
 
+// A fragment of X^T for a k-step of 16 rows of X: X is stored [k index][m index] (bf16, row
+// stride `stride` bytes); returns A(m0.., k0..) of the m16 x k16 product operand.
+__device__ __forceinline__ void load_a_trans(uint32_t base, int stride, int k0, int m0, int lane, uint32_t (&a)[4]) {
+    const int krow = k0 + (lane & 7) + ((lane >> 4) & 1) * 8;
+    const int mchunk = (m0 >> 3) + ((lane >> 3) & 1);
+    ldsm_x4_t(base + krow * stride + mchunk * 16, a[0], a[1], a[2], a[3]);
+}
+
+// A fragment (16 rows x 16 k) of a plain row-major bf16 tile with row stride `stride` bytes.
+__device__ __forceinline__ void load_a_plain(uint32_t base, int stride, int row0, int k0, int lane, uint32_t (&a)[4]) {
+    const int r = row0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    const int ch = (k0 >> 3) + (lane >> 4);
+    ldsm_x4(base + r * stride + ch * 16, a[0], a[1], a[2], a[3]);
+}
+
 }  // namespace bpt

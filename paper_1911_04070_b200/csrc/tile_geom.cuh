@@ -7,6 +7,11 @@
 namespace bpt {
 
 constexpr int kTileTokens = 64;  // tokens per CTA (4 warps x 16 rows)
+constexpr int kTileMaxK = 64;    // largest k the tiled kernels stage (k + 2 relation rows, k + 67 nodes per level)
+
+// The tiled kernels cover bf16, head size 64, at least one full tile of tokens and k <= 64;
+// everything else runs on the general row kernels.
+inline bool tile_path(int n, int k, int d, bool bf16) { return bf16 && d == 64 && n >= kTileTokens && k <= kTileMaxK; }
 
 // Number of levels that carry left / right contextual nodes for at least one token.
 inline void context_levels(const TreeParams& t, int* n_left, int* n_right) {
