@@ -1,14 +1,14 @@
 // Tiled backward for the token rows (arXiv 1911.04070: gradient of the Sec. 3.4 equation over
 // the contextual edges of Sec. 3.2.2), bf16, head size 64.
 //
-// One CTA = 64 consecutive tokens of one (batch entry, head), 4 warps.  As in the tiled forward
+// One CTA = 64 consecutive tokens of one (batch entry, head), 8 warps.  As in the tiled forward
 // the nodes a token attends at one (side, level) are one contiguous range, so per chunk the CTA
 // stages the union range of K and V rows once.  The token's self loop is folded into the
 // level-0 left chunk: node i follows its left neighbours directly, and the relation ids
 // self = 0, left(0, o) = 1 + o are consecutive, so the self loop is simply offset 0 of a range
 // that ends at the token itself.
 //
-//   phase 1 (a warp owns 16 query rows):  S = Q K^T + skewed Q R^T,  P = exp(S - lse),
+//   phase 1 (two warps share 16 query rows and take the key blocks in turn):  S = Q K^T + skewed Q R^T,  P = exp(S - lse),
 //            dP = dO V^T,  dS = P (dP - dO.O);  dQ += dS K + skew(dS) R;
 //            P, dS and the skewed dS (indexed by relation offset) go to shared memory as bf16
 //   phase 2 (a warp owns 16 staged key rows):  dK_part = dS^T Q,  dV_part = P^T dO for the
@@ -57,7 +57,30 @@ struct BwdTileSmem {
     static size_t bytes(int chunks) { return (size_t)fixed + (size_t)chunks * (kTileTokens * 8 + 8); }
 };
 
-__global__ void __launch_bounds__(128)
+constexpr int kBwdThreads = 256;  // 8 warps: two per group of 16 query rows
+
+// barrier of the two warps that share a group of query rows (ids 1..4; id 0 is __syncthreads)
+__device__ __forceinline__ void pair_barrier(int rg) { asm volatile("bar.sync %0, 64;" ::"r"(rg + 1) : "memory"); }
+
+struct ChunkGeom {
+    int side, level, n_l, id_base, rel_base, n_rel_c, base, kend, nr;
+};
+
+__device__ __forceinline__ ChunkGeom chunk_geom(const TreeParams& t, int n_left, int c, int2 cr) {
+    ChunkGeom gm;
+    gm.side = c >= n_left;
+    gm.level = gm.side ? c - n_left : c;
+    gm.n_l = t.n >> gm.level;
+    gm.id_base = node_id(t.n, gm.level, 0);
+    gm.rel_base = c == 0 ? 0 : (gm.side ? rel_right(t, gm.level, 0) : rel_left(t, gm.level, 0));
+    gm.n_rel_c = c == 0 ? t.k + 2 : t.k + 1;  // chunk 0 also holds r^self
+    gm.base = cr.x & ~15;
+    gm.kend = cr.y - gm.base;
+    gm.nr = min(kKvRows, (gm.kend + 1 + 31 + 15) & ~15);
+    return gm;
+}
+
+__global__ void __launch_bounds__(kBwdThreads)
 bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                 const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
@@ -82,6 +105,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
     int2* crange = bnd + chunks * kTileTokens;
 
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int rg = w & 3, half = w >> 2;  // row group (16 query rows) and which of its two warps
     const int g = lane >> 2, c2 = (lane & 3) * 2;
     const int tile = blockIdx.x, tiles = gridDim.x, t0 = tile * kTileTokens;
     const int pair = pair0 + blockIdx.y, b = pair / H, h = pair % H;
@@ -93,7 +117,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
     const float scale_log2e = scale * kLog2e;
 
     // ---- prologue: Q and dO tiles, out tile (into the K buffer) for the row term, row ranges ----
-    for (int idx = tid; idx < kTileTokens * 8; idx += 128) {
+    for (int idx = tid; idx < kTileTokens * 8; idx += kBwdThreads) {
         const int row = idx >> 3, ch = idx & 7;
         const size_t src = boff + (size_t)(t0 + row) * rs + ch * 8;
         cp_async16(q_u + tile_off(row, ch), q + src);
@@ -111,13 +135,13 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
     }
     cp_async_wait<0>();
     __syncthreads();
-    {   // delta_i = d_out_i . out_i: two threads per row
-        const int row = tid >> 1, half = tid & 1;
+    if (tid < 2 * kTileTokens) {   // delta_i = d_out_i . out_i: two threads per row
+        const int row = tid >> 1, hf = tid & 1;
         float acc = 0.f;
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
-            const uint4 a = *reinterpret_cast<const uint4*>(g_s + tile_off(row, half * 4 + ch));
-            const uint4 o = *reinterpret_cast<const uint4*>(k_s + tile_off(row, half * 4 + ch));
+            const uint4 a = *reinterpret_cast<const uint4*>(g_s + tile_off(row, hf * 4 + ch));
+            const uint4 o = *reinterpret_cast<const uint4*>(k_s + tile_off(row, hf * 4 + ch));
             const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, ow[4] = {o.x, o.y, o.z, o.w};
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
@@ -126,9 +150,9 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
             }
         }
         acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-        if (half == 0) delta_s[row] = acc;
+        if (hf == 0) delta_s[row] = acc;
     }
-    for (int c = w; c < chunks; c += 4) {
+    for (int c = w; c < chunks; c += kBwdThreads / 32) {
         const int2 a = rows_union(bnd + c * kTileTokens, 0, 32, lane);
         const int2 bb = rows_union(bnd + c * kTileTokens, 32, 32, lane);
         if (lane == 0) {
@@ -143,7 +167,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
         }
     }
 
-    const int r0 = w * 16;
+    const int r0 = rg * 16;
     uint32_t qa[4][4], ga[4][4];
     load_a_frags(q_u, r0, lane, qa);
     load_a_frags(g_u, r0, lane, ga);
@@ -151,55 +175,49 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt) { acc_q[nt][0] = acc_q[nt][1] = acc_q[nt][2] = acc_q[nt][3] = 0.f; }
 
-    float* qr_w = qr_s + w * 16 * kQrStride;
-    const int W = t.k + 1;
+    float* qr_w = qr_s + rg * 16 * kQrStride;
     float* slab_cta = slabs + ((size_t)blockIdx.y * tiles + tile) * plan.slab_row0[chunks] * 128;
     float* drel_cta = drel_part + ((size_t)blockIdx.y * tiles + tile) * chunks * plan.rel_rows * 64;
 
-    for (int c = 0; c < chunks; ++c) {
-        __syncthreads();  // previous chunk's tiles are free (and, first time, delta / crange are visible)
-        const int2 cr = crange[c];
-        if (cr.x > cr.y) {  // no token of the tile reaches this level: its d_rel partial is zero
-            float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)c * plan.rel_rows * 64);
-            for (int idx = tid; idx < plan.rel_rows * 16; idx += 128) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-            continue;
-        }
-        const int side = c >= n_left;
-        const int level = side ? c - n_left : c;
-        const int n_l = t.n >> level;
-        const int id_base = node_id(t.n, level, 0);
-        const int rel_base = c == 0 ? 0 : (side ? rel_right(t, level, 0) : rel_left(t, level, 0));
-        const int n_rel_c = c == 0 ? W + 1 : W;
-        const int base = cr.x & ~15;
-        const int kend = cr.y - base;
-        const int nr = min(kKvRows, (kend + 1 + 31 + 15) & ~15);
-
-        for (int idx = tid; idx < nr * 8; idx += 128) {
+    // K / V rows of the chunk's node range and its relation rows -> shared memory (async)
+    auto stage = [&](int c) {
+        const ChunkGeom gm = chunk_geom(t, n_left, c, crange[c]);
+        for (int idx = tid; idx < gm.nr * 8; idx += kBwdThreads) {
             const int row = idx >> 3, ch = idx & 7;
-            const int node = min(base + row, n_l - 1);
-            const size_t src = boff + (size_t)(id_base + node) * rs + ch * 8;
+            const int node = min(gm.base + row, gm.n_l - 1);
+            const size_t src = boff + (size_t)(gm.id_base + node) * rs + ch * 8;
             cp_async16(k_u + tile_off(row, ch), k + src);
             cp_async16(v_u + tile_off(row, ch), v + src);
         }
-        for (int idx = tid; idx < kRelRows * 8; idx += 128) {
+        for (int idx = tid; idx < kRelRows * 8; idx += kBwdThreads) {
             const int row = idx >> 3, ch = idx & 7;
-            if (row < n_rel_c) cp_async16(r_u + tile_off(row, ch), r + (size_t)(rel_base + row) * 64 + ch * 8);
+            if (row < gm.n_rel_c) cp_async16(r_u + tile_off(row, ch), r + (size_t)(gm.rel_base + row) * 64 + ch * 8);
             else *reinterpret_cast<uint4*>(r_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
         }
-        cp_async_commit();
-        for (int idx = tid; idx < kTileTokens * (kSkewStride / 16); idx += 128)
+    };
+
+    __syncthreads();  // delta and crange are visible; the out tile in the K buffer is consumed
+    stage(0);         // chunk 0 (left level 0 with the self loop) is never empty
+    cp_async_commit();
+
+    int c = 0;
+    while (c < chunks) {
+        for (int idx = tid; idx < kTileTokens * (kSkewStride / 16); idx += kBwdThreads)
             *reinterpret_cast<uint4*>(sk_s + idx * 16) = make_uint4(0, 0, 0, 0);
         cp_async_wait<0>();
         __syncthreads();
+        const int2 cr = crange[c];
+        const ChunkGeom gm = chunk_geom(t, n_left, c, cr);
+        const int side = gm.side, base = gm.base, kend = gm.kend, n_rel_c = gm.n_rel_c;
 
-        // ================= phase 1: this warp's 16 query rows =================
+        // ================= phase 1: 16 query rows per pair of warps, key blocks alternate =================
         const int2* bc = bnd + c * kTileTokens;
         const int2 wr = rows_union(bc, r0, 16, lane);
         const bool w_any = wr.x <= wr.y;
-        if (w_any) {  // Q R^T for the chunk's relation rows -> per-warp scratch
+        if (w_any) {  // Q R^T for the chunk's relation rows -> the row group's scratch
 #pragma unroll
             for (int np = 0; np < kRelRows / 16; ++np) {
-                if (np * 16 < n_rel_c) {
+                if (np * 16 < n_rel_c && (np & 1) == half) {
                     float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
@@ -219,17 +237,17 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 }
             }
         }
-        __syncwarp();
+        pair_barrier(rg);
 
         const int2 ba = bc[r0 + g], bb = bc[r0 + g + 8];
         const int lo_r[2] = {ba.x, bb.x}, hi_r[2] = {ba.y, bb.y};
         const float lse_r[2] = {lse_s[r0 + g], lse_s[r0 + g + 8]};
         const float del_r[2] = {delta_s[r0 + g], delta_s[r0 + g + 8]};
         const int w_lo = w_any ? wr.x - base : 1 << 30, w_hi = w_any ? wr.y - base : -1;
-        for (int kb = 0; kb <= kend; kb += 32) {
+        for (int kb = half * 32; kb <= kend; kb += 64) {
             unsigned char* p_row0 = p_s + (r0 + g) * kPStride + (kb + c2) * 2;
             unsigned char* d_row0 = ds_s + (r0 + g) * kPStride + (kb + c2) * 2;
-            if (kb + 31 < w_lo || kb > w_hi) {  // nothing of this warp's rows here: zeros for phase 2
+            if (kb + 31 < w_lo || kb > w_hi) {  // nothing of these rows here: zeros for phase 2
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     *reinterpret_cast<uint32_t*>(p_row0 + j * 16) = 0u;
@@ -298,11 +316,11 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 }
             }
         }
-        __syncwarp();
-        if (w_any) {  // dQ += skew(dS) R_chunk (this warp wrote its own 16 rows of the skew tile)
+        pair_barrier(rg);  // the group's rows of the skew tile are complete
+        if (w_any) {       // dQ += skew(dS) R_chunk, the k-steps shared out between the two warps
 #pragma unroll
             for (int kk = 0; kk < kRelRows / 16; ++kk) {
-                if (kk * 16 < n_rel_c) {
+                if (kk * 16 < n_rel_c && (kk & 1) == half) {
                     uint32_t a[4];
                     load_a_plain(sk_u, kSkewStride, r0, kk * 16, lane, a);
 #pragma unroll
@@ -315,86 +333,115 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 }
             }
         }
-        __syncthreads();
+        __syncthreads();  // P, dS and the skew tile are complete; K, V and R tiles are free
 
-        // ================= phase 2: this warp's key rows and relation offsets =================
-        const int n_jt = (kend >> 4) + 1;
-        for (int jt = w; jt < n_jt; jt += 4) {
-            float ak[8][4], av[8][4];
+        // next chunk that this tile reaches: its K / V / R rows arrive while phase 2 runs
+        int cn = c + 1;
+        while (cn < chunks && crange[cn].x > crange[cn].y) {  // a level no token of the tile reaches: zero d_rel partial
+            float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)cn * plan.rel_rows * 64);
+            for (int idx = tid; idx < plan.rel_rows * 16; idx += kBwdThreads) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+            ++cn;
+        }
+        if (cn < chunks) stage(cn);
+        cp_async_commit();
+
+        // ================= phase 2: key tiles (dk, dv partial rows) and offset tiles (d_rel partial) =================
+        const int n_jt = (kend >> 4) + 1, n_ot = plan.rel_rows >> 4;
+        for (int job = w; job < n_jt + n_ot; job += kBwdThreads / 32) {
+            if (job < n_jt) {
+                const int jt = job;
+                float ak[8][4], av[8][4];
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) {
-                ak[nt][0] = ak[nt][1] = ak[nt][2] = ak[nt][3] = 0.f;
-                av[nt][0] = av[nt][1] = av[nt][2] = av[nt][3] = 0.f;
-            }
-#pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                uint32_t a_ds[4], a_p[4];
-                load_a_trans(ds_u, kPStride, ks * 16, jt * 16, lane, a_ds);
-                load_a_trans(p_u, kPStride, ks * 16, jt * 16, lane, a_p);
-#pragma unroll
-                for (int np = 0; np < 4; ++np) {
-                    uint32_t bf[4];
-                    load_b_cols(q_u, ks * 16, np, lane, bf);
-                    mma_bf16(ak[np * 2], a_ds, bf[0], bf[1]);
-                    mma_bf16(ak[np * 2 + 1], a_ds, bf[2], bf[3]);
-                    load_b_cols(g_u, ks * 16, np, lane, bf);
-                    mma_bf16(av[np * 2], a_p, bf[0], bf[1]);
-                    mma_bf16(av[np * 2 + 1], a_p, bf[2], bf[3]);
+                for (int nt = 0; nt < 8; ++nt) {
+                    ak[nt][0] = ak[nt][1] = ak[nt][2] = ak[nt][3] = 0.f;
+                    av[nt][0] = av[nt][1] = av[nt][2] = av[nt][3] = 0.f;
                 }
-            }
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                const int m = base + jt * 16 + g + hh * 8;
-                if (m >= cr.x && m <= cr.y) {
-                    float* dst = slab_cta + (size_t)(plan.slab_row0[c] + m - cr.x) * 128 + c2;
+                for (int ks = 0; ks < 4; ++ks) {
+                    uint32_t a_ds[4], a_p[4];
+                    load_a_trans(ds_u, kPStride, ks * 16, jt * 16, lane, a_ds);
+                    load_a_trans(p_u, kPStride, ks * 16, jt * 16, lane, a_p);
 #pragma unroll
-                    for (int nt = 0; nt < 8; ++nt) {
-                        *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ak[nt][hh * 2], ak[nt][hh * 2 + 1]);
-                        *reinterpret_cast<float2*>(dst + 64 + nt * 8) = make_float2(av[nt][hh * 2], av[nt][hh * 2 + 1]);
+                    for (int np = 0; np < 4; ++np) {
+                        uint32_t bf[4];
+                        load_b_cols(q_u, ks * 16, np, lane, bf);
+                        mma_bf16(ak[np * 2], a_ds, bf[0], bf[1]);
+                        mma_bf16(ak[np * 2 + 1], a_ds, bf[2], bf[3]);
+                        load_b_cols(g_u, ks * 16, np, lane, bf);
+                        mma_bf16(av[np * 2], a_p, bf[0], bf[1]);
+                        mma_bf16(av[np * 2 + 1], a_p, bf[2], bf[3]);
                     }
                 }
-            }
-        }
-        const int n_ot = plan.rel_rows >> 4;
-        for (int ot = 3 - w; ot < n_ot; ot += 4) {  // warps in reverse order: warp 3 has the fewest key tiles
-            float ar[8][4];
 #pragma unroll
-            for (int nt = 0; nt < 8; ++nt) { ar[nt][0] = ar[nt][1] = ar[nt][2] = ar[nt][3] = 0.f; }
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int m = base + jt * 16 + g + hh * 8;
+                    if (m >= cr.x && m <= cr.y) {
+                        float* dst = slab_cta + (size_t)(plan.slab_row0[c] + m - cr.x) * 128 + c2;
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                uint32_t a[4];
-                load_a_trans(sk_u, kSkewStride, ks * 16, ot * 16, lane, a);
+                        for (int nt = 0; nt < 8; ++nt) {
+                            *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ak[nt][hh * 2], ak[nt][hh * 2 + 1]);
+                            *reinterpret_cast<float2*>(dst + 64 + nt * 8) = make_float2(av[nt][hh * 2], av[nt][hh * 2 + 1]);
+                        }
+                    }
+                }
+            } else {
+                const int ot = job - n_jt;
+                float ar[8][4];
 #pragma unroll
-                for (int np = 0; np < 4; ++np) {
-                    uint32_t bf[4];
-                    load_b_cols(q_u, ks * 16, np, lane, bf);
-                    mma_bf16(ar[np * 2], a, bf[0], bf[1]);
-                    mma_bf16(ar[np * 2 + 1], a, bf[2], bf[3]);
+                for (int nt = 0; nt < 8; ++nt) { ar[nt][0] = ar[nt][1] = ar[nt][2] = ar[nt][3] = 0.f; }
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    uint32_t a[4];
+                    load_a_trans(sk_u, kSkewStride, ks * 16, ot * 16, lane, a);
+#pragma unroll
+                    for (int np = 0; np < 4; ++np) {
+                        uint32_t bf[4];
+                        load_b_cols(q_u, ks * 16, np, lane, bf);
+                        mma_bf16(ar[np * 2], a, bf[0], bf[1]);
+                        mma_bf16(ar[np * 2 + 1], a, bf[2], bf[3]);
+                    }
+                }
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int o = ot * 16 + g + hh * 8;
+                    float* dst = drel_cta + ((size_t)c * plan.rel_rows + o) * 64 + c2;
+#pragma unroll
+                    for (int nt = 0; nt < 8; ++nt)
+                        *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ar[nt][hh * 2], ar[nt][hh * 2 + 1]);
                 }
             }
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                const int o = ot * 16 + g + hh * 8;
-                float* dst = drel_cta + ((size_t)c * plan.rel_rows + o) * 64 + c2;
-#pragma unroll
-                for (int nt = 0; nt < 8; ++nt)
-                    *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ar[nt][hh * 2], ar[nt][hh * 2 + 1]);
-            }
         }
+        __syncthreads();  // P, dS and skew tiles are free again
+        c = cn;
     }
 
-    // ---- epilogue: dq = scale * acc, rounded once to bf16, coalesced stores through the Q tile ----
-    __syncthreads();
+    // ---- epilogue: the two warps' dq parts are added (second warp's part through shared memory), ----
+    // ---- dq = scale * sum, rounded once to bf16, coalesced stores through the Q tile              ----
+    float* red = reinterpret_cast<float*>(p_s) + rg * 16 * 64;  // [16 rows][64] per row group
+    if (half == 1) {
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-        *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g, nt) + c2 * 2) = pack_bf16(acc_q[nt][0] * scale, acc_q[nt][1] * scale);
-        *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g + 8, nt) + c2 * 2) = pack_bf16(acc_q[nt][2] * scale, acc_q[nt][3] * scale);
+        for (int nt = 0; nt < 8; ++nt) {
+            *reinterpret_cast<float2*>(red + g * 64 + nt * 8 + c2) = make_float2(acc_q[nt][0], acc_q[nt][1]);
+            *reinterpret_cast<float2*>(red + (g + 8) * 64 + nt * 8 + c2) = make_float2(acc_q[nt][2], acc_q[nt][3]);
+        }
     }
-    __syncwarp();
-    for (int idx = lane; idx < 16 * 8; idx += 32) {
-        const int row = r0 + (idx >> 3), ch = idx & 7;
-        *reinterpret_cast<uint4*>(dq + boff + (size_t)(t0 + row) * rs + ch * 8) =
-            *reinterpret_cast<const uint4*>(q_s + tile_off(row, ch));
+    __syncthreads();
+    if (half == 0) {
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            const float2 x = *reinterpret_cast<const float2*>(red + g * 64 + nt * 8 + c2);
+            const float2 y = *reinterpret_cast<const float2*>(red + (g + 8) * 64 + nt * 8 + c2);
+            *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g, nt) + c2 * 2) =
+                pack_bf16((acc_q[nt][0] + x.x) * scale, (acc_q[nt][1] + x.y) * scale);
+            *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g + 8, nt) + c2 * 2) =
+                pack_bf16((acc_q[nt][2] + y.x) * scale, (acc_q[nt][3] + y.y) * scale);
+        }
+        __syncwarp();
+        for (int idx = lane; idx < 16 * 8; idx += 32) {
+            const int row = r0 + (idx >> 3), ch = idx & 7;
+            *reinterpret_cast<uint4*>(dq + boff + (size_t)(t0 + row) * rs + ch * 8) =
+                *reinterpret_cast<const uint4*>(q_s + tile_off(row, ch));
+        }
     }
 }
 
@@ -558,7 +605,7 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
         // span rows: dq of the spans and, per token, the affiliated edges' share of dk / dv
         const bpt_status s = launch_bwd_span(p, pair0, np, ws.ext_dq, ws.aff_slab);
         if (s != BPT_OK) return s;
-        bwd_tile_kernel<<<dim3(tiles, np), 128, smem, p.stream>>>(
+        bwd_tile_kernel<<<dim3(tiles, np), kBwdThreads, smem, p.stream>>>(
             t, plan, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
             (const __nv_bfloat16*)p.rel_emb, (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out,
             (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale);
