@@ -73,6 +73,13 @@ SMALL = [
     (512, 16, 1, 1, 4, 64, False),
     (1024, 1, 0, 1, 8, 32, True),
     (2048, 3, 3, 1, 2, 64, True),
+    # tiled tensor-core path (bf16, d = 64, n >= 64, k <= 64): its corner cases
+    (64, 64, 0, 1, 1, 64, True),       # one tile, no outer ancestors, k = n
+    (64, 1, 1, 3, 2, 64, True),        # one tile, thinnest graph, left only
+    (128, 64, 0, 2, 2, 64, True),      # widest staging (k = 64), both sides, two tiles
+    (256, 33, 1, 1, 3, 64, True),      # odd k, left only
+    (512, 63, 2, 1, 2, 64, True),      # Algorithm-1 graph, k + 1 = 64 relation rows exactly
+    (4096, 64, 0, 1, 1, 64, True),     # k = 64 on both sides over 64 tiles
 ]
 
 
