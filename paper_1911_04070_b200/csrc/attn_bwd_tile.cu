@@ -60,7 +60,14 @@ struct BwdTileSmem {
 constexpr int kBwdThreads = 256;  // 8 warps: two per group of 16 query rows
 
 // barrier of the two warps that share a group of query rows (ids 1..4; id 0 is __syncthreads)
-__device__ __forceinline__ void pair_barrier(int rg) { asm volatile("bar.sync %0, 64;" ::"r"(rg + 1) : "memory"); }
+__device__ __forceinline__ void pair_barrier(int rg) {
+    switch (rg) {
+        case 0: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
+        case 1: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
+        case 2: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
+        default: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
+    }
+}
 
 struct ChunkGeom {
     int side, level, n_l, id_base, rel_base, n_rel_c, base, kend, nr;
