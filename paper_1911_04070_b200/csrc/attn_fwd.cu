@@ -2,6 +2,8 @@
 // relative-position term of Sec. 3.4).  General row kernel: one CTA per (batch, node,
 // head group); its warps take the row's edges in turns, each keeps an online softmax in
 // registers, and the per-warp states are merged in a fixed order through shared memory.
+#include <cstdlib>
+
 #include "bpt_internal.cuh"
 #include "row_map.cuh"
 #include "tile_geom.cuh"
@@ -141,19 +143,32 @@ static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows) {
 }
 
 bpt_status launch_fwd_tile(const AttnProblem& p);
+bool fwd_tc5_eligible(const AttnProblem& p);
+bpt_status launch_fwd_tc5(const AttnProblem& p, int* status);
 size_t fwd_span_workspace_bytes(const TreeParams& t, int B, int H);
 bpt_status launch_fwd_span(const AttnProblem& p);
+
+constexpr size_t kStatusBytes = 256;  // device status word at the end of the forward workspace
+
+static size_t span_ws_bytes(const TreeParams& t, int B, int H) { return (fwd_span_workspace_bytes(t, B, H) + 255) & ~(size_t)255; }
 
 size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype) {
     if (!tile_path(g.dims.n, g.dims.k, d, dtype == BPT_BF16)) return 0;
     TreeParams t;
     tree_params_from_dims(g.dims, &t);
-    return fwd_span_workspace_bytes(t, B, H);
+    return span_ws_bytes(t, B, H) + kStatusBytes;
+}
+
+// BPT_FWD_TOKENS=mma selects the warp-level (mma.sync) token kernel where the tensor-memory one would run.
+static bool want_tc5() {
+    static const bool v = [] { const char* e = getenv("BPT_FWD_TOKENS"); return !(e && e[0] == 'm'); }();
+    return v;
 }
 
 bpt_status launch_fwd(const AttnProblem& p) {
     if (tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16)) {  // token rows and span rows on the tensor cores
-        const bpt_status s = launch_fwd_tile(p);
+        int* status = reinterpret_cast<int*>(static_cast<char*>(p.workspace) + span_ws_bytes(p.tree, p.B, p.H));
+        const bpt_status s = (want_tc5() && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, status) : launch_fwd_tile(p);
         return s != BPT_OK ? s : launch_fwd_span(p);
     }
     const int row0 = 0, nrows = p.g->dims.n_nodes;

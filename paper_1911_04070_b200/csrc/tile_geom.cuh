@@ -23,16 +23,17 @@ inline void context_levels(const TreeParams& t, int* n_left, int* n_right) {
     *n_right = nr;
 }
 
-// bnd[c * 64 + r] = (first, last) node index at the chunk's level that token t0 + r attends;
+// bnd[c * TILE + r] = (first, last) node index at the chunk's level that token t0 + r attends;
 // chunks 0..n_left-1 are the left levels, n_left..n_left+n_right-1 the right levels.
 // Rows that do not reach a level get an empty range that keeps the bounds monotone in r.
+template <int TILE = kTileTokens>
 __device__ __forceinline__ void fill_row_bounds(const TreeParams& t, int t0, int r, int n_left, int n_right, int2* bnd) {
     {
         LeftWalk w(t, t0 + r);
         for (int c = 0; c < n_left; ++c) {
             int2 v = make_int2(0, -1);
             if (w.valid()) { v = make_int2(w.lo, w.hi); w.next(); }
-            bnd[c * kTileTokens + r] = v;
+            bnd[c * TILE + r] = v;
         }
     }
     {
@@ -41,7 +42,7 @@ __device__ __forceinline__ void fill_row_bounds(const TreeParams& t, int t0, int
             const int n_l = t.n >> c;
             int2 v = make_int2(n_l, n_l - 1);
             if (w.valid()) { v = make_int2(w.lo, w.hi); w.next(); }
-            bnd[(n_left + c) * kTileTokens + r] = v;
+            bnd[(n_left + c) * TILE + r] = v;
         }
     }
 }
