@@ -159,9 +159,11 @@ size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dt
     return span_ws_bytes(t, B, H) + kStatusBytes;
 }
 
-// BPT_FWD_TOKENS=mma selects the warp-level (mma.sync) token kernel where the tensor-memory one would run.
+// Two kernels cover the token rows: the warp-level one (mma.sync, 64-token tiles) and the tensor-memory
+// one (tcgen05, 128-token tiles).  The faster one on the measured workloads is the default;
+// BPT_FWD_TOKENS=tc5 / =mma in the environment picks the other for comparison runs.
 static bool want_tc5() {
-    static const bool v = [] { const char* e = getenv("BPT_FWD_TOKENS"); return !(e && e[0] == 'm'); }();
+    static const bool v = [] { const char* e = getenv("BPT_FWD_TOKENS"); return e && e[0] == 't'; }();
     return v;
 }
 
