@@ -17,10 +17,16 @@
 // which each thread adds (its 32 channels) to the running output row with the usual rescale.
 // The self loop is offset 0 of the level-0 left chunk, as in the tiled backward.
 //
-// Pipeline: at the one block-wide barrier of a chunk (P complete) the elected thread issues
-// O_chunk and at once QR and S of the next chunk, whose K / R / V rows were fetched while the
-// softmax ran (K and R buffers are free as soon as S is done, V has two buffers); O_chunk is
-// collected at the start of the next chunk.  Every wait on an mbarrier has an iteration limit.
+// Warp roles: eight softmax warps and one driver warp.  The driver's elected thread brings the K, V and R
+// rows in with TMA (cp.async.bulk.tensor, 16-row boxes straight into the swizzled layout the
+// tensor core reads) and issues every MMA; mbarriers carry all hand-offs (rows landed -> driver,
+// S / QR done and O_chunk done -> softmax threads, P complete -> driver), so the softmax code has
+// no block-wide barrier.  QR and S of the next chunk are issued as soon as P of this one is
+// complete, the next K / R rows are fetched as soon as S is done (single buffers) and the next V
+// rows into the other of two buffers; O_chunk is collected at the start of the next chunk.
+// Every mbarrier wait gives up after about a second and the kernel then winds down.
+#include <cuda.h>
+
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
 #include "tc5_tools.cuh"
@@ -33,7 +39,8 @@ namespace {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTcTokens = 128;
-constexpr int kTcThreads = 256;
+constexpr int kTcSoftmaxThreads = 256;             // two per token row
+constexpr int kTcThreads = kTcSoftmaxThreads + 32;  // + the driver warp (TMA and MMA issue)
 constexpr int kTcKvRows = 208;    // staged K / V rows per chunk: 128 + 64 + 2 nodes, rounded up to 16
 constexpr int kTcRelRows = 80;    // relation rows per chunk (k + 2 <= 66), rounded up to 16
 constexpr int kTcBiasRows = 68;   // offsets kept in the bias table
@@ -47,9 +54,9 @@ struct FwdTcSmem {
     static constexpr int r_off = v_off + 2 * kTcKvRows * 128;
     static constexpr int p_off = r_off + kTcRelRows * 128;               // 4 key blocks of [128 rows][128 B]
     static constexpr int bias_off = p_off + 4 * kTcTokens * 128;         // [68 offsets][128 rows] fp32
-    static constexpr int misc_off = bias_off + kTcBiasRows * kTcTokens * 4;  // 2 mbarriers, tensor-memory slot, abort flag
-    static constexpr int xch_off = misc_off + 64;                        // [2 halves][128 rows] fp32 exchange
-    static constexpr int bnd_off = xch_off + 2 * kTcTokens * 4;          // [chunks][128] short2, then [chunks] int2
+    static constexpr int misc_off = bias_off + kTcBiasRows * kTcTokens * 4;  // 6 mbarriers, tensor-memory slot, abort flag
+    static constexpr int xch_off = misc_off + 64;                        // [2 halves][128 rows] fp32 exchange + the same of give-up flags
+    static constexpr int bnd_off = xch_off + 4 * kTcTokens * 4;          // [chunks][128] short2, then [chunks] int2
     static size_t bytes(int chunks) { return (size_t)bnd_off + (size_t)chunks * (kTcTokens * 4 + 8) + 1024; }
 };
 static_assert(FwdTcSmem::k_off % 1024 == 0 && FwdTcSmem::v_off % 1024 == 0 && FwdTcSmem::r_off % 1024 == 0 &&
@@ -76,7 +83,8 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
                const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
                __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int* __restrict__ status,
-               int H, float scale_log2e) {
+               int H, float scale_log2e, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_r) {
     extern __shared__ unsigned char smem_raw[];
     // the swizzle pattern is a function of the address bits, so the tiles must start 1024-aligned
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -85,9 +93,10 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
     unsigned char* r_s = smem + FwdTcSmem::r_off;
     float* bias_s = reinterpret_cast<float*>(smem + FwdTcSmem::bias_off);
     uint64_t* mbar = reinterpret_cast<uint64_t*>(smem + FwdTcSmem::misc_off);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 2);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 6);
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* xch_s = reinterpret_cast<float*>(smem + FwdTcSmem::xch_off);
+    int* dead_s = reinterpret_cast<int*>(xch_s + 2 * kTcTokens);
     short2* bnd = reinterpret_cast<short2*>(smem + FwdTcSmem::bnd_off);  // row ranges relative to the chunk's first node
     const int chunks = n_left + n_right;
     int2* crange = reinterpret_cast<int2*>(bnd + chunks * kTcTokens);
@@ -100,7 +109,9 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
     const size_t boff = (size_t)b * N_nodes * rs + (size_t)h * 64;
     const uint32_t q_u = smem_u32(q_s), k_u = smem_u32(smem + FwdTcSmem::k_off), v_u = smem_u32(smem + FwdTcSmem::v_off),
                    r_u = smem_u32(r_s), p_u = smem_u32(p_s);
-    const uint32_t mbar_s = smem_u32(&mbar[0]), mbar_o = smem_u32(&mbar[1]);
+    // S / QR done, O_chunk done, K + R rows landed, V rows landed (two buffers), P complete
+    const uint32_t mbar_s = smem_u32(&mbar[0]), mbar_o = smem_u32(&mbar[1]), mbar_kr = smem_u32(&mbar[2]),
+                   mbar_v0 = smem_u32(&mbar[3]), mbar_v1 = smem_u32(&mbar[4]), mbar_p = smem_u32(&mbar[5]);
 
     // ---- prologue: Q tile, row ranges, barriers, tensor memory ----
     for (int idx = tid; idx < kTcTokens * 8; idx += kTcThreads) {
@@ -118,6 +129,10 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
     if (tid == 0) {
         tc5::mbar_init(mbar_s, 1);
         tc5::mbar_init(mbar_o, 1);
+        tc5::mbar_init(mbar_kr, 1);
+        tc5::mbar_init(mbar_v0, 1);
+        tc5::mbar_init(mbar_v1, 1);
+        tc5::mbar_init(mbar_p, kTcSoftmaxThreads);
         tc5::mbar_init_fence();
         *abort_s = 0;
     }
@@ -146,7 +161,6 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
     }
     __syncthreads();
 
-    // K / R / V rows of a chunk -> shared memory, asynchronously
     auto geom = [&](int c, int& level, int& side, int& base, int& n_cols) {
         const int2 cr = crange[c];
         side = c >= n_left;
@@ -154,202 +168,227 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
         base = cr.x;
         n_cols = (cr.y - cr.x + 1 + 15) & ~15;
     };
-    auto stage = [&](int c, int vbuf) {
-        int level, side, base, n_cols;
-        geom(c, level, side, base, n_cols);
-        const int n_l = t.n >> level, id_base = node_id(t.n, level, 0);
-        const int rel_base = c == 0 ? 0 : (side ? rel_right(t, level, 0) : rel_left(t, level, 0));
-        const int n_rel_c = c == 0 ? t.k + 2 : t.k + 1;
-        const uint32_t vb_u = v_u + vbuf * (kTcKvRows * 128);
-        for (int idx = tid; idx < n_cols * 8; idx += kTcThreads) {
-            const int rr = idx >> 3, ch = idx & 7;
-            const int node = min(base + rr, n_l - 1);  // rows past the range repeat a real row: finite values
-            const size_t src = boff + (size_t)(id_base + node) * rs + ch * 8;
-            cp_async16(k_u + tile_off(rr, ch), k + src);
-            cp_async16(vb_u + tile_off(rr, ch), v + src);
-        }
-        for (int idx = tid; idx < kTcRelRows * 8; idx += kTcThreads) {
-            const int rr = idx >> 3, ch = idx & 7;
-            if (rr < n_rel_c) cp_async16(r_u + tile_off(rr, ch), r + (size_t)(rel_base + rr) * 64 + ch * 8);
-            else *reinterpret_cast<uint4*>(r_s + tile_off(rr, ch)) = make_uint4(0, 0, 0, 0);
-        }
-        cp_async_commit();
-    };
-    // QR and S of chunk c (elected thread)
-    auto issue_s = [&](int c) {
-        int level, side, base, n_cols;
-        geom(c, level, side, base, n_cols);
-        const uint32_t id_qr = tc5::instr_desc(kTcTokens, kTcRelRows, 0, 0), id_s = tc5::instr_desc(kTcTokens, n_cols, 0, 0);
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-            tc5::mma(tbase + kColQR, tc5::desc_k_major(q_u + ks * 32), tc5::desc_k_major(r_u + ks * 32), id_qr, ks > 0);
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-            tc5::mma(tbase + kColS, tc5::desc_k_major(q_u + ks * 32), tc5::desc_k_major(k_u + ks * 32), id_s, ks > 0);
-        tc5::commit(mbar_s);
-    };
-
-    float m_run = -INFINITY, l_run = 0.f, corr_prev = 1.f, o[32];  // this thread's 32 channels of the row
-#pragma unroll
-    for (int j = 0; j < 32; ++j) o[j] = 0.f;
-    uint32_t ph_s = 0, ph_o = 0;
-    bool o_pending = false;
-    // O_chunk of the previous chunk -> running output (rescaled by that chunk's correction)
-    auto collect_o = [&]() {
-        if (!tc5::mbar_wait(mbar_o, ph_o)) *abort_s = 1;
-        ph_o ^= 1;
-        tc5::fence_after_sync();
-        uint32_t x[32];
-        tc5::tmem_ld32(tbase + lane_base + kColO + half * 32, x);
-        tc5::tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) o[j] = fmaf(o[j], corr_prev, __uint_as_float(x[j]));
-    };
-
-    stage(0, 0);  // chunk 0 (left level 0 with the self loop) is never empty
-    cp_async_wait<0>();
-    tc5::fence_async_smem();
-    tc5::fence_before_sync();
-    __syncthreads();
-    if (tid == 0) { tc5::fence_after_sync(); issue_s(0); }
-
-    int c = 0, it = 0;
-    while (c < chunks) {
-        int level, side, base, n_cols;
-        geom(c, level, side, base, n_cols);
-        if (!tc5::mbar_wait(mbar_s, ph_s)) *abort_s = 1;  // S and QR of this chunk are in tensor memory
-        ph_s ^= 1;
-        tc5::fence_after_sync();
-        if (o_pending) collect_o();  // also: the other V buffer and the P tile are free now
-
-        int cn = c + 1;  // next chunk this tile reaches: its rows arrive while the softmax runs
+    auto next_chunk = [&](int c) {  // next chunk this tile reaches
+        int cn = c + 1;
         while (cn < chunks && crange[cn].x > crange[cn].y) ++cn;
-        if (cn < chunks) stage(cn, (it + 1) & 1);
+        return cn;
+    };
 
-        // ---- bias row -> table [offset][row]; the two threads of a row share the offsets ----
-        {
+    if (w == kTcSoftmaxThreads / 32) {
+        // =============== driver: one thread moves the tiles (TMA) and issues every MMA ===============
+        if (lane == 0) {
+            // K and R rows of chunk c (16 rows per copy; rows past the range are real rows of later
+            // nodes / relations or, past the end of the tensor, zeros: finite either way)
+            auto load_kr = [&](int c) {
+                int level, side, base, n_cols;
+                geom(c, level, side, base, n_cols);
+                const int node0 = node_id(t.n, level, 0) + base;
+                const int rel_base = c == 0 ? 0 : (side ? rel_right(t, level, 0) : rel_left(t, level, 0));
+                tc5::mbar_expect_tx(mbar_kr, (uint32_t)(n_cols / 16 + kTcRelRows / 16) * 2048u);
+                for (int j = 0; j < n_cols / 16; ++j) tc5::tma_load_4d(k_u + j * 2048, &tm_k, 0, h, node0 + 16 * j, b, mbar_kr);
+                for (int j = 0; j < kTcRelRows / 16; ++j) tc5::tma_load_2d(r_u + j * 2048, &tm_r, 0, rel_base + 16 * j, mbar_kr);
+            };
+            auto load_v = [&](int c, int buf) {
+                int level, side, base, n_cols;
+                geom(c, level, side, base, n_cols);
+                const int node0 = node_id(t.n, level, 0) + base;
+                const uint32_t bar = buf ? mbar_v1 : mbar_v0;
+                tc5::mbar_expect_tx(bar, (uint32_t)(n_cols / 16) * 2048u);
+                for (int j = 0; j < n_cols / 16; ++j)
+                    tc5::tma_load_4d(v_u + buf * (kTcKvRows * 128) + j * 2048, &tm_v, 0, h, node0 + 16 * j, b, bar);
+            };
+            auto issue_s = [&](int c) {  // QR and S of chunk c
+                int level, side, base, n_cols;
+                geom(c, level, side, base, n_cols);
+                const uint32_t id_qr = tc5::instr_desc(kTcTokens, kTcRelRows, 0, 0), id_s = tc5::instr_desc(kTcTokens, n_cols, 0, 0);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    tc5::mma(tbase + kColQR, tc5::desc_k_major(q_u + ks * 32), tc5::desc_k_major(r_u + ks * 32), id_qr, ks > 0);
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks)
+                    tc5::mma(tbase + kColS, tc5::desc_k_major(q_u + ks * 32), tc5::desc_k_major(k_u + ks * 32), id_s, ks > 0);
+                tc5::commit(mbar_s);
+            };
+            uint32_t ph_kr = 0, ph_v[2] = {0, 0}, ph_p = 0, ph_s = 0, ph_o = 0;
+            bool ok = true;
+            load_kr(0);  // chunk 0 (left level 0 with the self loop) is never empty
+            load_v(0, 0);
+            ok = tc5::mbar_wait(mbar_kr, ph_kr); ph_kr ^= 1;
+            tc5::fence_after_sync();
+            if (ok) issue_s(0);
+            int c = 0, it = 0;
+            while (ok && c < chunks && !*abort_s) {
+                int level, side, base, n_cols;
+                geom(c, level, side, base, n_cols);
+                const int cn = next_chunk(c);
+                ok = tc5::mbar_wait(mbar_s, ph_s); ph_s ^= 1;         // S, QR done: K and R buffers are free
+                if (ok && cn < chunks) load_kr(cn);
+                if (ok && it > 0) { ok = tc5::mbar_wait(mbar_o, ph_o); ph_o ^= 1; }  // O_chunk of the chunk before: other V buffer free
+                if (ok && cn < chunks) load_v(cn, (it + 1) & 1);
+                if (ok) { ok = tc5::mbar_wait(mbar_p, ph_p); ph_p ^= 1; }            // P complete; S, QR, O_chunk have been read
+                if (ok) { ok = tc5::mbar_wait((it & 1) ? mbar_v1 : mbar_v0, ph_v[it & 1]); ph_v[it & 1] ^= 1; }
+                if (!ok) break;
+                tc5::fence_after_sync();
+                const uint32_t id_o = tc5::instr_desc(kTcTokens, 64, 0, 1);
+                const uint32_t vb_u = v_u + (it & 1) * (kTcKvRows * 128);
+                for (int kk = 0; kk < (n_cols >> 4); ++kk)
+                    tc5::mma(tbase + kColO, tc5::desc_k_major(p_u + (kk >> 2) * (kTcTokens * 128) + (kk & 3) * 32),
+                             tc5::desc_mn_major(vb_u + kk * 2048), id_o, kk > 0);
+                tc5::commit(mbar_o);
+                if (cn < chunks) {
+                    ok = tc5::mbar_wait(mbar_kr, ph_kr); ph_kr ^= 1;
+                    if (ok) issue_s(cn);
+                }
+                c = cn;
+                ++it;
+            }
+            if (!ok) *abort_s = 1;
+        }
+    } else {
+        // =============== softmax: two threads per token row ===============
+        float m_run = -INFINITY, l_run = 0.f, corr_prev = 1.f, o[32];  // this thread's 32 channels of the row
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o[j] = 0.f;
+        uint32_t ph_s = 0, ph_o = 0;
+        bool o_pending = false;
+        // O_chunk of the previous chunk -> running output (rescaled by that chunk's correction)
+        auto collect_o = [&]() {
+            if (!tc5::mbar_wait(mbar_o, ph_o)) *abort_s = 1;
+            ph_o ^= 1;
+            tc5::fence_after_sync();
             uint32_t x[32];
-            tc5::tmem_ld32(tbase + lane_base + kColQR + half * 32, x);
+            tc5::tmem_ld32(tbase + lane_base + kColO + half * 32, x);
             tc5::tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) bias_s[(half * 32 + j) * kTcTokens + row] = __uint_as_float(x[j]) * scale_log2e;
-            if (half == 0) {  // offsets 64 .. 67 (k + 2 <= 66 are used)
-                uint32_t y[16];
-                tc5::tmem_ld16(tbase + lane_base + kColQR + 64, y);
+            for (int j = 0; j < 32; ++j) o[j] = fmaf(o[j], corr_prev, __uint_as_float(x[j]));
+        };
+
+        int c = 0;
+        while (c < chunks) {
+            int level, side, base, n_cols;
+            geom(c, level, side, base, n_cols);
+            if (!tc5::mbar_wait(mbar_s, ph_s)) *abort_s = 1;  // S and QR of this chunk are in tensor memory
+            ph_s ^= 1;
+            tc5::fence_after_sync();
+            if (o_pending) collect_o();  // also: the P tile is free now
+            const int dead = *abort_s;   // some wait gave up: leave, but together with the row's other thread (below)
+
+            // ---- bias row -> table [offset][row]; the two threads of a row share the offsets ----
+            {
+                uint32_t x[32];
+                tc5::tmem_ld32(tbase + lane_base + kColQR + half * 32, x);
                 tc5::tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < kTcBiasRows - 64; ++j) bias_s[(64 + j) * kTcTokens + row] = __uint_as_float(y[j]) * scale_log2e;
-            }
-        }
-
-        // ---- this thread's half of the row's part of S ----
-        const short2 my = bnd[c * kTcTokens + row];
-        int wlo = my.x <= my.y ? my.x : 0x7fff, whi = my.x <= my.y ? my.y : -1;
+                for (int j = 0; j < 32; ++j) bias_s[(half * 32 + j) * kTcTokens + row] = __uint_as_float(x[j]) * scale_log2e;
+                if (half == 0) {  // offsets 64 .. 67 (k + 2 <= 66 are used)
+                    uint32_t y[16];
+                    tc5::tmem_ld16(tbase + lane_base + kColQR + 64, y);
+                    tc5::tmem_ld_wait();
 #pragma unroll
-        for (int sh = 16; sh > 0; sh >>= 1) {
-            wlo = min(wlo, __shfl_xor_sync(0xffffffffu, wlo, sh));
-            whi = max(whi, __shfl_xor_sync(0xffffffffu, whi, sh));
-        }
-        const bool w_any = wlo <= whi;
-        const int c0 = w_any ? (wlo & ~7) : 0;
-        const int npieces = w_any ? min(kTcPieces, ((whi - c0) >> 5) + 1) : 0;
-        uint32_t sv[kTcPieces][16];
-#pragma unroll
-        for (int p = 0; p < kTcPieces; ++p)
-            if (p < npieces) tc5::tmem_ld16(tbase + lane_base + kColS + c0 + p * 32 + half * 16, sv[p]);
-        tc5::tmem_ld_wait();
-        quad_barrier(quad);  // the row's bias values are all in the table
-
-        const int cnt = max(my.y - my.x + 1, 0);
-        const int a = my.x - c0 - half * 16;  // column, relative to this thread's first one, of the row's first node
-        // offset of column e: right side e - a, left side (cnt - 1) - (e - a): one pointer and a signed stride
-        const int sgn = side ? kTcTokens : -kTcTokens;
-        const float* bptr = bias_s + row + (side ? -a : (cnt - 1 + a)) * kTcTokens;
-        float mx = -INFINITY;
-#pragma unroll
-        for (int p = 0; p < kTcPieces; ++p) {
-            if (p < npieces) {
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int e = p * 32 + j;
-                    const bool ok = (unsigned)(e - a) < (unsigned)cnt;
-                    float val = -INFINITY;
-                    if (ok) val = fmaf(__uint_as_float(sv[p][j]), scale_log2e, bptr[e * sgn]);
-                    sv[p][j] = __float_as_uint(val);
-                    mx = fmaxf(mx, val);
+                    for (int j = 0; j < kTcBiasRows - 64; ++j) bias_s[(64 + j) * kTcTokens + row] = __uint_as_float(y[j]) * scale_log2e;
                 }
             }
-        }
-        xch_s[half * kTcTokens + row] = mx;
-        quad_barrier(quad);
-        const float m_new = fmaxf(m_run, fmaxf(mx, xch_s[(half ^ 1) * kTcTokens + row]));
-        const float m_ref = m_new == -INFINITY ? 0.f : m_new;
-        const float corr = ex2(m_run - m_ref);
-        m_run = m_new;
-        float l_add = 0.f;
-        const int ch0 = c0 >> 3, n_ch = n_cols >> 3;
+
+            // ---- this thread's half of the row's part of S ----
+            const short2 my = bnd[c * kTcTokens + row];
+            int wlo = my.x <= my.y ? my.x : 0x7fff, whi = my.x <= my.y ? my.y : -1;
 #pragma unroll
-        for (int p = 0; p < kTcPieces; ++p) {
-            if (p < npieces) {
+            for (int sh = 16; sh > 0; sh >>= 1) {
+                wlo = min(wlo, __shfl_xor_sync(0xffffffffu, wlo, sh));
+                whi = max(whi, __shfl_xor_sync(0xffffffffu, whi, sh));
+            }
+            const bool w_any = wlo <= whi;
+            const int c0 = w_any ? (wlo & ~7) : 0;
+            const int npieces = w_any ? min(kTcPieces, ((whi - c0) >> 5) + 1) : 0;
+            uint32_t sv[kTcPieces][16];
 #pragma unroll
-                for (int qd = 0; qd < 2; ++qd) {
-                    uint32_t pk[4];
+            for (int p = 0; p < kTcPieces; ++p)
+                if (p < npieces) tc5::tmem_ld16(tbase + lane_base + kColS + c0 + p * 32 + half * 16, sv[p]);
+            tc5::tmem_ld_wait();
+            quad_barrier(quad);  // the row's bias values are all in the table
+
+            const int cnt = max(my.y - my.x + 1, 0);
+            const int a = my.x - c0 - half * 16;  // column, relative to this thread's first one, of the row's first node
+            // offset of column e: right side e - a, left side (cnt - 1) - (e - a): one pointer and a signed stride
+            const int sgn = side ? kTcTokens : -kTcTokens;
+            const float* bptr = bias_s + row + (side ? -a : (cnt - 1 + a)) * kTcTokens;
+            float mx = -INFINITY;
 #pragma unroll
-                    for (int x = 0; x < 4; ++x) {
-                        const float p0 = ex2(__uint_as_float(sv[p][qd * 8 + 2 * x]) - m_ref);
-                        const float p1 = ex2(__uint_as_float(sv[p][qd * 8 + 2 * x + 1]) - m_ref);
-                        l_add += p0 + p1;
-                        pk[x] = pack_bf16(p0, p1);
+            for (int p = 0; p < kTcPieces; ++p) {
+                if (p < npieces) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int e = p * 32 + j;
+                        const bool in = (unsigned)(e - a) < (unsigned)cnt;
+                        float val = -INFINITY;
+                        if (in) val = fmaf(__uint_as_float(sv[p][j]), scale_log2e, bptr[e * sgn]);
+                        sv[p][j] = __float_as_uint(val);
+                        mx = fmaxf(mx, val);
                     }
-                    const int ci = ch0 + p * 4 + half * 2 + qd;  // 16-byte chunk (8 keys) of the P row
-                    if (ci < n_ch)
-                        *reinterpret_cast<uint4*>(p_s + (ci >> 3) * (kTcTokens * 128) + tile_off(row, ci & 7)) =
-                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
             }
-        }
-        l_run = fmaf(l_run, corr, l_add);
-        corr_prev = corr;
-        for (int ci = half; ci < n_ch; ci += 2)  // the rest of the row is zero (the two threads take alternate chunks)
-            if (ci < ch0 || ci >= ch0 + npieces * 4)
-                *reinterpret_cast<uint4*>(p_s + (ci >> 3) * (kTcTokens * 128) + tile_off(row, ci & 7)) = make_uint4(0, 0, 0, 0);
+            xch_s[half * kTcTokens + row] = mx;
+            dead_s[half * kTcTokens + row] = dead;
+            quad_barrier(quad);
+            // the 64 threads of a lane quadrant share barriers and warp-wide loads: they leave as one
+            if (__any_sync(0xffffffffu, dead | dead_s[(half ^ 1) * kTcTokens + row])) break;
+            const float m_new = fmaxf(m_run, fmaxf(mx, xch_s[(half ^ 1) * kTcTokens + row]));
+            const float m_ref = m_new == -INFINITY ? 0.f : m_new;
+            const float corr = ex2(m_run - m_ref);
+            m_run = m_new;
+            float l_add = 0.f;
+            const int ch0 = c0 >> 3, n_ch = n_cols >> 3;
+#pragma unroll
+            for (int p = 0; p < kTcPieces; ++p) {
+                if (p < npieces) {
+#pragma unroll
+                    for (int qd = 0; qd < 2; ++qd) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            const float p0 = ex2(__uint_as_float(sv[p][qd * 8 + 2 * x]) - m_ref);
+                            const float p1 = ex2(__uint_as_float(sv[p][qd * 8 + 2 * x + 1]) - m_ref);
+                            l_add += p0 + p1;
+                            pk[x] = pack_bf16(p0, p1);
+                        }
+                        const int ci = ch0 + p * 4 + half * 2 + qd;  // 16-byte chunk (8 keys) of the P row
+                        if (ci < n_ch)
+                            *reinterpret_cast<uint4*>(p_s + (ci >> 3) * (kTcTokens * 128) + tile_off(row, ci & 7)) =
+                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+            }
+            l_run = fmaf(l_run, corr, l_add);
+            corr_prev = corr;
+            for (int ci = half; ci < n_ch; ci += 2)  // the rest of the row is zero (the two threads take alternate chunks)
+                if (ci < ch0 || ci >= ch0 + npieces * 4)
+                    *reinterpret_cast<uint4*>(p_s + (ci >> 3) * (kTcTokens * 128) + tile_off(row, ci & 7)) = make_uint4(0, 0, 0, 0);
 
-        cp_async_wait<0>();  // next chunk's rows (this thread's copies)
-        tc5::fence_async_smem();
-        tc5::fence_before_sync();
-        __syncthreads();  // P is complete, the next chunk's rows are in place, S / QR / O_chunk have been read
-        if (tid == 0) {
-            tc5::fence_after_sync();
-            const uint32_t id_o = tc5::instr_desc(kTcTokens, 64, 0, 1);
-            const uint32_t vb_u = v_u + (it & 1) * (kTcKvRows * 128);
-            for (int kk = 0; kk < (n_cols >> 4); ++kk)
-                tc5::mma(tbase + kColO, tc5::desc_k_major(p_u + (kk >> 2) * (kTcTokens * 128) + (kk & 3) * 32),
-                         tc5::desc_mn_major(vb_u + kk * 2048), id_o, kk > 0);
-            tc5::commit(mbar_o);
-            if (cn < chunks && !*abort_s) issue_s(cn);
+            tc5::fence_async_smem();   // P was written with ordinary stores and is read by the tensor core
+            tc5::fence_before_sync();
+            tc5::mbar_arrive(mbar_p);  // this thread's part of P is in place and its tensor-memory reads are done
+            o_pending = true;
+            c = next_chunk(c);
         }
-        o_pending = true;
-        if (*abort_s) break;  // set before the barrier by whoever gave up on a wait
-        c = cn;
-        ++it;
+        if (o_pending && !*abort_s) collect_o();
+
+        // ---- row sums of the two threads, normalise, round once to bf16 into the Q tile ----
+        xch_s[half * kTcTokens + row] = l_run;
+        quad_barrier(quad);
+        const float l_all = l_run + xch_s[(half ^ 1) * kTcTokens + row];
+        const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) pk[x] = pack_bf16(o[ch * 8 + 2 * x] * inv, o[ch * 8 + 2 * x + 1] * inv);
+            *reinterpret_cast<uint4*>(q_s + tile_off(row, half * 4 + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+        if (half == 0) lse[((size_t)b * N_nodes + t0 + row) * H + h] = (m_run + log2f(l_all)) * kLn2;
     }
-    if (o_pending) collect_o();
 
-    // ---- epilogue: row sums of the two threads, normalise, round once to bf16, coalesced stores ----
-    cp_async_wait<0>();
-    xch_s[half * kTcTokens + row] = l_run;
+    // ---- epilogue: coalesced stores of the output tile; tensor memory back ----
     tc5::fence_before_sync();
-    __syncthreads();
-    const float l_all = l_run + xch_s[(half ^ 1) * kTcTokens + row];
-    const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
-#pragma unroll
-    for (int ch = 0; ch < 4; ++ch) {
-        uint32_t pk[4];
-#pragma unroll
-        for (int x = 0; x < 4; ++x) pk[x] = pack_bf16(o[ch * 8 + 2 * x] * inv, o[ch * 8 + 2 * x + 1] * inv);
-        *reinterpret_cast<uint4*>(q_s + tile_off(row, half * 4 + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-    }
-    if (half == 0) lse[((size_t)b * N_nodes + t0 + row) * H + h] = (m_run + log2f(l_all)) * kLn2;
     __syncthreads();
     for (int idx = tid; idx < kTcTokens * 8; idx += kTcThreads) {
         const int rr = idx >> 3, ch = idx & 7;
@@ -362,8 +401,49 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
 
 }  // namespace
 
+namespace {
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime (the library does not link libcuda).
+EncodeTiledFn encode_tiled() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess ||
+            qr != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Map over a [B, N, H, 64] bf16 tensor: a box is 16 consecutive nodes of one (batch entry, head), 128-byte swizzle.
+bool node_rows_map(CUtensorMap* m, const void* base, int B, int N, int H) {
+    const cuuint64_t dims[4] = {64, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {128, (cuuint64_t)H * 128, (cuuint64_t)N * H * 128};
+    const cuuint32_t box[4] = {64, 1, 16, 1}, estr[4] = {1, 1, 1, 1};
+    return encode_tiled()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// Map over the [n_rel, 64] relation table: a box is 16 consecutive relations.
+bool rel_rows_map(CUtensorMap* m, const void* base, int n_rel) {
+    const cuuint64_t dims[2] = {64, (cuuint64_t)n_rel};
+    const cuuint64_t strides[1] = {128};
+    const cuuint32_t box[2] = {64, 16}, estr[2] = {1, 1};
+    return encode_tiled()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 // The tensor-memory kernel takes whole tiles of 128 tokens.
 bool fwd_tc5_eligible(const AttnProblem& p) {
+    if (!encode_tiled()) return false;
     if (!tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16) || p.tree.n < kTcTokens) return false;
     int n_left, n_right;
     context_levels(p.tree, &n_left, &n_right);
@@ -378,11 +458,16 @@ bpt_status launch_fwd_tc5(const AttnProblem& p, int* status) {
     if (smem > 227 * 1024 || p.H > 65535 || p.B > 65535) return BPT_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(fwd_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return BPT_ERR_CUDA;
+    alignas(64) CUtensorMap tm_k, tm_v, tm_r;
+    const int N = 2 * p.tree.n - 1;
+    if (!encode_tiled() || !node_rows_map(&tm_k, p.k, p.B, N, p.H) || !node_rows_map(&tm_v, p.v, p.B, N, p.H) ||
+        !rel_rows_map(&tm_r, p.rel_emb, p.g->dims.n_rel))
+        return BPT_ERR_CUDA;
     const dim3 grid(p.tree.n / kTcTokens, p.H, p.B);
     fwd_tc5_kernel<<<grid, kTcThreads, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q,
                                                          (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
                                                          (const __nv_bfloat16*)p.rel_emb, (__nv_bfloat16*)p.out, p.lse,
-                                                         status, p.H, p.scale * kLog2e);
+                                                         status, p.H, p.scale * kLog2e, tm_k, tm_v, tm_r);
     trace_mark(p.stream, "fwd_tc5");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }
