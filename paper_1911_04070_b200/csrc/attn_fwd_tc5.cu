@@ -3,18 +3,18 @@
 // bf16, head size 64.
 //
 // One CTA = 128 consecutive tokens of one (batch entry, head) = the 128 lanes of tensor memory,
-// 256 threads: two threads per token row (warps w and w + 4 read the same lane quadrant), each
-// taking half of the columns.  Per (side, level) chunk the union node range of the tile (at most
+// four threads per token row (warps w, w + 4, w + 8, w + 12 read the same lane quadrant), each
+// taking a quarter of the columns, plus a driver warp.  Per (side, level) chunk the union node range of the tile (at most
 // 128 / 2^level + k + 2 nodes) is staged once in shared memory, and one elected thread issues
 //     QR = Q R_chunk^T   (128 x 80)        -- the relative-position terms of every offset
 //     S  = Q K_range^T   (128 x N, N <= 208)
 // into tensor memory.  The row's bias values go to a shared table indexed [offset][row], so that
 // the per-row shift between node index and offset is plain address arithmetic; the part of S that
-// covers the warp's rows is read into registers (16 columns of each 32-column piece per thread)
+// covers the warp's rows is read into registers (8 columns of each 32-column piece per thread)
 // and the row does its masked softmax update in one sweep -- the softmax code issues no
 // tensor-core instruction.  P goes to shared memory as the K-major A operand of
 //     O_chunk = P V_range (128 x 64),
-// which each thread adds (its 32 channels) to the running output row with the usual rescale.
+// which each thread adds (its 16 channels) to the running output row with the usual rescale.
 // The self loop is offset 0 of the level-0 left chunk, as in the tiled backward.
 //
 // Warp roles: eight softmax warps and one driver warp.  The driver's elected thread brings the K, V and R
@@ -39,7 +39,8 @@ namespace {
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kTcTokens = 128;
-constexpr int kTcSoftmaxThreads = 256;             // two per token row
+constexpr int kTpr = 4;                             // threads per token row
+constexpr int kTcSoftmaxThreads = kTcTokens * kTpr;
 constexpr int kTcThreads = kTcSoftmaxThreads + 32;  // + the driver warp (TMA and MMA issue)
 constexpr int kTcKvRows = 208;    // staged K / V rows per chunk: 128 + 64 + 2 nodes, rounded up to 16
 constexpr int kTcRelRows = 80;    // relation rows per chunk (k + 2 <= 66), rounded up to 16
@@ -54,9 +55,9 @@ struct FwdTcSmem {
     static constexpr int r_off = v_off + 2 * kTcKvRows * 128;
     static constexpr int p_off = r_off + kTcRelRows * 128;               // 4 key blocks of [128 rows][128 B]
     static constexpr int bias_off = p_off + 4 * kTcTokens * 128;         // [68 offsets][128 rows] fp32
-    static constexpr int misc_off = bias_off + kTcBiasRows * kTcTokens * 4;  // 6 mbarriers, tensor-memory slot, abort flag
+    static constexpr int misc_off = bias_off + kTcBiasRows * kTcTokens * 4;  // 7 mbarriers, tensor-memory slot, abort flag
     static constexpr int xch_off = misc_off + 64;                        // [2 halves][128 rows] fp32 exchange + the same of give-up flags
-    static constexpr int bnd_off = xch_off + 4 * kTcTokens * 4;          // [chunks][128] short2, then [chunks] int2
+    static constexpr int bnd_off = xch_off + 2 * kTpr * kTcTokens * 4;          // [chunks][128] short2, then [chunks] int2
     static size_t bytes(int chunks) { return (size_t)bnd_off + (size_t)chunks * (kTcTokens * 4 + 8) + 1024; }
 };
 static_assert(FwdTcSmem::k_off % 1024 == 0 && FwdTcSmem::v_off % 1024 == 0 && FwdTcSmem::r_off % 1024 == 0 &&
@@ -68,13 +69,13 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// barrier of the two warps that share a lane quadrant (ids 1..4; id 0 is __syncthreads)
+// barrier of the kTpr warps that share a lane quadrant (ids 1..4; id 0 is __syncthreads)
 __device__ __forceinline__ void quad_barrier(int quad) {
     switch (quad) {
-        case 0: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
-        case 1: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
-        case 2: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
-        default: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
+        case 0: asm volatile("bar.sync 1, %0;" ::"n"(32 * kTpr) : "memory"); break;
+        case 1: asm volatile("bar.sync 2, %0;" ::"n"(32 * kTpr) : "memory"); break;
+        case 2: asm volatile("bar.sync 3, %0;" ::"n"(32 * kTpr) : "memory"); break;
+        default: asm volatile("bar.sync 4, %0;" ::"n"(32 * kTpr) : "memory"); break;
     }
 }
 
@@ -93,25 +94,26 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
     unsigned char* r_s = smem + FwdTcSmem::r_off;
     float* bias_s = reinterpret_cast<float*>(smem + FwdTcSmem::bias_off);
     uint64_t* mbar = reinterpret_cast<uint64_t*>(smem + FwdTcSmem::misc_off);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 6);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(mbar + 7);
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* xch_s = reinterpret_cast<float*>(smem + FwdTcSmem::xch_off);
-    int* dead_s = reinterpret_cast<int*>(xch_s + 2 * kTcTokens);
+    int* dead_s = reinterpret_cast<int*>(xch_s + kTpr * kTcTokens);
     short2* bnd = reinterpret_cast<short2*>(smem + FwdTcSmem::bnd_off);  // row ranges relative to the chunk's first node
     const int chunks = n_left + n_right;
     int2* crange = reinterpret_cast<int2*>(bnd + chunks * kTcTokens);
 
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int quad = w & 3, half = w >> 2, row = quad * 32 + lane;
+    const int quad = w & 3, part = w >> 2, row = quad * 32 + lane;  // part: which share of the row's columns / channels
     const int t0 = blockIdx.x * kTcTokens, h = blockIdx.y, b = blockIdx.z;
     const int N_nodes = 2 * t.n - 1;
     const size_t rs = (size_t)H * 64;
     const size_t boff = (size_t)b * N_nodes * rs + (size_t)h * 64;
     const uint32_t q_u = smem_u32(q_s), k_u = smem_u32(smem + FwdTcSmem::k_off), v_u = smem_u32(smem + FwdTcSmem::v_off),
                    r_u = smem_u32(r_s), p_u = smem_u32(p_s);
-    // S / QR done, O_chunk done, K + R rows landed, V rows landed (two buffers), P complete
+    // S / QR done, O_chunk done, K + R rows landed, V rows landed (two buffers), P complete, S / QR read
     const uint32_t mbar_s = smem_u32(&mbar[0]), mbar_o = smem_u32(&mbar[1]), mbar_kr = smem_u32(&mbar[2]),
-                   mbar_v0 = smem_u32(&mbar[3]), mbar_v1 = smem_u32(&mbar[4]), mbar_p = smem_u32(&mbar[5]);
+                   mbar_v0 = smem_u32(&mbar[3]), mbar_v1 = smem_u32(&mbar[4]), mbar_p = smem_u32(&mbar[5]),
+                   mbar_r = smem_u32(&mbar[6]);
 
     // ---- prologue: Q tile, row ranges, barriers, tensor memory ----
     for (int idx = tid; idx < kTcTokens * 8; idx += kTcThreads) {
@@ -133,6 +135,7 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
         tc5::mbar_init(mbar_v0, 1);
         tc5::mbar_init(mbar_v1, 1);
         tc5::mbar_init(mbar_p, kTcSoftmaxThreads);
+        tc5::mbar_init(mbar_r, kTcSoftmaxThreads);
         tc5::mbar_init_fence();
         *abort_s = 0;
     }
@@ -209,7 +212,7 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
                     tc5::mma(tbase + kColS, tc5::desc_k_major(q_u + ks * 32), tc5::desc_k_major(k_u + ks * 32), id_s, ks > 0);
                 tc5::commit(mbar_s);
             };
-            uint32_t ph_kr = 0, ph_v[2] = {0, 0}, ph_p = 0, ph_s = 0, ph_o = 0;
+            uint32_t ph_kr = 0, ph_v[2] = {0, 0}, ph_p = 0, ph_s = 0, ph_o = 0, ph_r = 0;
             bool ok = true;
             load_kr(0);  // chunk 0 (left level 0 with the self loop) is never empty
             load_v(0, 0);
@@ -223,9 +226,15 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
                 const int cn = next_chunk(c);
                 ok = tc5::mbar_wait(mbar_s, ph_s); ph_s ^= 1;         // S, QR done: K and R buffers are free
                 if (ok && cn < chunks) load_kr(cn);
+                if (ok && cn < chunks) {
+                    // S and QR of the next chunk as soon as every thread holds its part of this chunk's S and QR
+                    ok = tc5::mbar_wait(mbar_r, ph_r); ph_r ^= 1;
+                    if (ok) { ok = tc5::mbar_wait(mbar_kr, ph_kr); ph_kr ^= 1; }
+                    if (ok) { tc5::fence_after_sync(); issue_s(cn); }
+                }
                 if (ok && it > 0) { ok = tc5::mbar_wait(mbar_o, ph_o); ph_o ^= 1; }  // O_chunk of the chunk before: other V buffer free
                 if (ok && cn < chunks) load_v(cn, (it + 1) & 1);
-                if (ok) { ok = tc5::mbar_wait(mbar_p, ph_p); ph_p ^= 1; }            // P complete; S, QR, O_chunk have been read
+                if (ok) { ok = tc5::mbar_wait(mbar_p, ph_p); ph_p ^= 1; }            // P complete, O_chunk has been read
                 if (ok) { ok = tc5::mbar_wait((it & 1) ? mbar_v1 : mbar_v0, ph_v[it & 1]); ph_v[it & 1] ^= 1; }
                 if (!ok) break;
                 tc5::fence_after_sync();
@@ -235,10 +244,6 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
                     tc5::mma(tbase + kColO, tc5::desc_k_major(p_u + (kk >> 2) * (kTcTokens * 128) + (kk & 3) * 32),
                              tc5::desc_mn_major(vb_u + kk * 2048), id_o, kk > 0);
                 tc5::commit(mbar_o);
-                if (cn < chunks) {
-                    ok = tc5::mbar_wait(mbar_kr, ph_kr); ph_kr ^= 1;
-                    if (ok) issue_s(cn);
-                }
                 c = cn;
                 ++it;
             }
@@ -246,9 +251,10 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
         }
     } else {
         // =============== softmax: two threads per token row ===============
-        float m_run = -INFINITY, l_run = 0.f, corr_prev = 1.f, o[32];  // this thread's 32 channels of the row
+        constexpr int kCols = 32 / kTpr, kChan = 64 / kTpr;  // columns per 32-column piece and output channels of one thread
+        float m_run = -INFINITY, l_run = 0.f, corr_prev = 1.f, o[kChan];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) o[j] = 0.f;
+        for (int j = 0; j < kChan; ++j) o[j] = 0.f;
         uint32_t ph_s = 0, ph_o = 0;
         bool o_pending = false;
         // O_chunk of the previous chunk -> running output (rescaled by that chunk's correction)
@@ -256,11 +262,11 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
             if (!tc5::mbar_wait(mbar_o, ph_o)) *abort_s = 1;
             ph_o ^= 1;
             tc5::fence_after_sync();
-            uint32_t x[32];
-            tc5::tmem_ld32(tbase + lane_base + kColO + half * 32, x);
+            uint32_t x[kChan];
+            tc5::tmem_ld16(tbase + lane_base + kColO + part * kChan, x);
             tc5::tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = fmaf(o[j], corr_prev, __uint_as_float(x[j]));
+            for (int j = 0; j < kChan; ++j) o[j] = fmaf(o[j], corr_prev, __uint_as_float(x[j]));
         };
 
         int c = 0;
@@ -270,26 +276,24 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
             if (!tc5::mbar_wait(mbar_s, ph_s)) *abort_s = 1;  // S and QR of this chunk are in tensor memory
             ph_s ^= 1;
             tc5::fence_after_sync();
-            if (o_pending) collect_o();  // also: the P tile is free now
             const int dead = *abort_s;   // some wait gave up: leave, but together with the row's other thread (below)
 
-            // ---- bias row -> table [offset][row]; the two threads of a row share the offsets ----
+            // ---- bias row -> table [offset][row]; the threads of a row share the offsets ----
             {
-                uint32_t x[32];
-                tc5::tmem_ld32(tbase + lane_base + kColQR + half * 32, x);
+                uint32_t x[16];
+                tc5::tmem_ld16(tbase + lane_base + kColQR + part * 16, x);
                 tc5::tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) bias_s[(half * 32 + j) * kTcTokens + row] = __uint_as_float(x[j]) * scale_log2e;
-                if (half == 0) {  // offsets 64 .. 67 (k + 2 <= 66 are used)
-                    uint32_t y[16];
-                    tc5::tmem_ld16(tbase + lane_base + kColQR + 64, y);
+                for (int j = 0; j < 16; ++j) bias_s[(part * 16 + j) * kTcTokens + row] = __uint_as_float(x[j]) * scale_log2e;
+                if (part == 0) {  // offsets 64 .. 67 (k + 2 <= 66 are used)
+                    tc5::tmem_ld16(tbase + lane_base + kColQR + 64, x);
                     tc5::tmem_ld_wait();
 #pragma unroll
-                    for (int j = 0; j < kTcBiasRows - 64; ++j) bias_s[(64 + j) * kTcTokens + row] = __uint_as_float(y[j]) * scale_log2e;
+                    for (int j = 0; j < kTcBiasRows - 64; ++j) bias_s[(64 + j) * kTcTokens + row] = __uint_as_float(x[j]) * scale_log2e;
                 }
             }
 
-            // ---- this thread's half of the row's part of S ----
+            // ---- this thread's share of the row's part of S ----
             const short2 my = bnd[c * kTcTokens + row];
             int wlo = my.x <= my.y ? my.x : 0x7fff, whi = my.x <= my.y ? my.y : -1;
 #pragma unroll
@@ -300,67 +304,75 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
             const bool w_any = wlo <= whi;
             const int c0 = w_any ? (wlo & ~7) : 0;
             const int npieces = w_any ? min(kTcPieces, ((whi - c0) >> 5) + 1) : 0;
-            uint32_t sv[kTcPieces][16];
+            uint32_t sv[kTcPieces][kCols];
 #pragma unroll
             for (int p = 0; p < kTcPieces; ++p)
-                if (p < npieces) tc5::tmem_ld16(tbase + lane_base + kColS + c0 + p * 32 + half * 16, sv[p]);
+                if (p < npieces) tc5::tmem_ld8(tbase + lane_base + kColS + c0 + p * 32 + part * kCols, sv[p]);
             tc5::tmem_ld_wait();
-            quad_barrier(quad);  // the row's bias values are all in the table
+            tc5::fence_before_sync();
+            tc5::mbar_arrive(mbar_r);  // this thread holds its part of S and QR: the driver may overwrite them
+            quad_barrier(quad);        // the row's bias values are all in the table
 
             const int cnt = max(my.y - my.x + 1, 0);
-            const int a = my.x - c0 - half * 16;  // column, relative to this thread's first one, of the row's first node
+            const int a = my.x - c0 - part * kCols;  // column, relative to this thread's first one, of the row's first node
             // offset of column e: right side e - a, left side (cnt - 1) - (e - a): one pointer and a signed stride
             const int sgn = side ? kTcTokens : -kTcTokens;
             const float* bptr = bias_s + row + (side ? -a : (cnt - 1 + a)) * kTcTokens;
-            float mx = -INFINITY;
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // independent chains
 #pragma unroll
             for (int p = 0; p < kTcPieces; ++p) {
                 if (p < npieces) {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
+                    for (int j = 0; j < kCols; ++j) {
                         const int e = p * 32 + j;
                         const bool in = (unsigned)(e - a) < (unsigned)cnt;
                         float val = -INFINITY;
                         if (in) val = fmaf(__uint_as_float(sv[p][j]), scale_log2e, bptr[e * sgn]);
                         sv[p][j] = __float_as_uint(val);
-                        mx = fmaxf(mx, val);
+                        mx4[j & 3] = fmaxf(mx4[j & 3], val);
                     }
                 }
             }
-            xch_s[half * kTcTokens + row] = mx;
-            dead_s[half * kTcTokens + row] = dead;
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+            xch_s[part * kTcTokens + row] = mx;
+            dead_s[part * kTcTokens + row] = dead;
             quad_barrier(quad);
-            // the 64 threads of a lane quadrant share barriers and warp-wide loads: they leave as one
-            if (__any_sync(0xffffffffu, dead | dead_s[(half ^ 1) * kTcTokens + row])) break;
-            const float m_new = fmaxf(m_run, fmaxf(mx, xch_s[(half ^ 1) * kTcTokens + row]));
+            // the threads of a lane quadrant share barriers and warp-wide loads: they leave as one
+            int dead_row = 0;
+            float mx_row = -INFINITY;
+#pragma unroll
+            for (int x = 0; x < kTpr; ++x) {
+                dead_row |= dead_s[x * kTcTokens + row];
+                mx_row = fmaxf(mx_row, xch_s[x * kTcTokens + row]);
+            }
+            if (__any_sync(0xffffffffu, dead_row)) break;
+            const float m_new = fmaxf(m_run, mx_row);
             const float m_ref = m_new == -INFINITY ? 0.f : m_new;
             const float corr = ex2(m_run - m_ref);
             m_run = m_new;
-            float l_add = 0.f;
+            if (o_pending) collect_o();  // O_chunk of the chunk before; the P tile is free after it
+            float l4[4] = {0.f, 0.f, 0.f, 0.f};
             const int ch0 = c0 >> 3, n_ch = n_cols >> 3;
 #pragma unroll
             for (int p = 0; p < kTcPieces; ++p) {
                 if (p < npieces) {
+                    uint32_t pk[4];
 #pragma unroll
-                    for (int qd = 0; qd < 2; ++qd) {
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int x = 0; x < 4; ++x) {
-                            const float p0 = ex2(__uint_as_float(sv[p][qd * 8 + 2 * x]) - m_ref);
-                            const float p1 = ex2(__uint_as_float(sv[p][qd * 8 + 2 * x + 1]) - m_ref);
-                            l_add += p0 + p1;
-                            pk[x] = pack_bf16(p0, p1);
-                        }
-                        const int ci = ch0 + p * 4 + half * 2 + qd;  // 16-byte chunk (8 keys) of the P row
-                        if (ci < n_ch)
-                            *reinterpret_cast<uint4*>(p_s + (ci >> 3) * (kTcTokens * 128) + tile_off(row, ci & 7)) =
-                                make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    for (int x = 0; x < 4; ++x) {
+                        const float p0 = ex2(__uint_as_float(sv[p][2 * x]) - m_ref);
+                        const float p1 = ex2(__uint_as_float(sv[p][2 * x + 1]) - m_ref);
+                        l4[x] += p0 + p1;
+                        pk[x] = pack_bf16(p0, p1);
                     }
+                    const int ci = ch0 + p * 4 + part;  // 16-byte chunk (8 keys) of the P row
+                    if (ci < n_ch)
+                        *reinterpret_cast<uint4*>(p_s + (ci >> 3) * (kTcTokens * 128) + tile_off(row, ci & 7)) =
+                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
                 }
             }
-            l_run = fmaf(l_run, corr, l_add);
+            l_run = fmaf(l_run, corr, (l4[0] + l4[1]) + (l4[2] + l4[3]));
             corr_prev = corr;
-            for (int ci = half; ci < n_ch; ci += 2)  // the rest of the row is zero (the two threads take alternate chunks)
+            for (int ci = part; ci < n_ch; ci += kTpr)  // the rest of the row is zero (the row's threads take chunks in turn)
                 if (ci < ch0 || ci >= ch0 + npieces * 4)
                     *reinterpret_cast<uint4*>(p_s + (ci >> 3) * (kTcTokens * 128) + tile_off(row, ci & 7)) = make_uint4(0, 0, 0, 0);
 
@@ -372,19 +384,21 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
         }
         if (o_pending && !*abort_s) collect_o();
 
-        // ---- row sums of the two threads, normalise, round once to bf16 into the Q tile ----
-        xch_s[half * kTcTokens + row] = l_run;
+        // ---- row sums of the row's threads, normalise, round once to bf16 into the Q tile ----
+        xch_s[part * kTcTokens + row] = l_run;
         quad_barrier(quad);
-        const float l_all = l_run + xch_s[(half ^ 1) * kTcTokens + row];
+        float l_all = 0.f;
+#pragma unroll
+        for (int x = 0; x < kTpr; ++x) l_all += xch_s[x * kTcTokens + row];
         const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
+        for (int ch = 0; ch < kChan / 8; ++ch) {
             uint32_t pk[4];
 #pragma unroll
             for (int x = 0; x < 4; ++x) pk[x] = pack_bf16(o[ch * 8 + 2 * x] * inv, o[ch * 8 + 2 * x + 1] * inv);
-            *reinterpret_cast<uint4*>(q_s + tile_off(row, half * 4 + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            *reinterpret_cast<uint4*>(q_s + tile_off(row, part * (kChan / 8) + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
-        if (half == 0) lse[((size_t)b * N_nodes + t0 + row) * H + h] = (m_run + log2f(l_all)) * kLn2;
+        if (part == 0) lse[((size_t)b * N_nodes + t0 + row) * H + h] = (m_run + log2f(l_all)) * kLn2;
     }
 
     // ---- epilogue: coalesced stores of the output tile; tensor memory back ----
