@@ -160,17 +160,18 @@ size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dt
 }
 
 // Two kernels cover the token rows: the warp-level one (mma.sync, 64-token tiles) and the tensor-memory
-// one (tcgen05, 128-token tiles).  The faster one on the measured workloads is the default;
-// BPT_FWD_TOKENS=tc5 / =mma in the environment picks the other for comparison runs.
-static bool want_tc5() {
-    static const bool v = [] { const char* e = getenv("BPT_FWD_TOKENS"); return e && e[0] == 't'; }();
-    return v;
+// one (tcgen05 + TMA, 128-token tiles).  The second wins where a chunk holds enough nodes per token to
+// pay for its per-chunk hand-offs (measured at n = 8192: 0.32 against 0.34 ms at k = 64, 0.33 against 0.30 ms at
+// k = 48, 0.34 against 0.26 ms at k = 16; 6 to 12 % faster at k = 64 for n = 4096 .. 65536), so it takes k >= 56.  BPT_FWD_TOKENS=tc5 / =mma in the environment forces one of them for comparison runs.
+static bool want_tc5(int k) {
+    static const int forced = [] { const char* e = getenv("BPT_FWD_TOKENS"); return !e ? 0 : (e[0] == 't' ? 1 : (e[0] == 'm' ? 2 : 0)); }();
+    return forced == 1 || (forced == 0 && k >= 56);
 }
 
 bpt_status launch_fwd(const AttnProblem& p) {
     if (tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16)) {  // token rows and span rows on the tensor cores
         int* status = reinterpret_cast<int*>(static_cast<char*>(p.workspace) + span_ws_bytes(p.tree, p.B, p.H));
-        const bpt_status s = (want_tc5() && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, status) : launch_fwd_tile(p);
+        const bpt_status s = (want_tc5(p.tree.k) && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, status) : launch_fwd_tile(p);
         return s != BPT_OK ? s : launch_fwd_span(p);
     }
     const int row0 = 0, nrows = p.g->dims.n_nodes;

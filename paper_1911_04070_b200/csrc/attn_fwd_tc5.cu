@@ -171,6 +171,7 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
         base = cr.x;
         n_cols = (cr.y - cr.x + 1 + 15) & ~15;
     };
+    const int rel_cols = (t.k + 2 + 15) & ~15;  // relation rows (offsets) a chunk can use, in whole 16-row boxes
     auto next_chunk = [&](int c) {  // next chunk this tile reaches
         int cn = c + 1;
         while (cn < chunks && crange[cn].x > crange[cn].y) ++cn;
@@ -187,9 +188,9 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
                 geom(c, level, side, base, n_cols);
                 const int node0 = node_id(t.n, level, 0) + base;
                 const int rel_base = c == 0 ? 0 : (side ? rel_right(t, level, 0) : rel_left(t, level, 0));
-                tc5::mbar_expect_tx(mbar_kr, (uint32_t)(n_cols / 16 + kTcRelRows / 16) * 2048u);
+                tc5::mbar_expect_tx(mbar_kr, (uint32_t)(n_cols / 16 + rel_cols / 16) * 2048u);
                 for (int j = 0; j < n_cols / 16; ++j) tc5::tma_load_4d(k_u + j * 2048, &tm_k, 0, h, node0 + 16 * j, b, mbar_kr);
-                for (int j = 0; j < kTcRelRows / 16; ++j) tc5::tma_load_2d(r_u + j * 2048, &tm_r, 0, rel_base + 16 * j, mbar_kr);
+                for (int j = 0; j < rel_cols / 16; ++j) tc5::tma_load_2d(r_u + j * 2048, &tm_r, 0, rel_base + 16 * j, mbar_kr);
             };
             auto load_v = [&](int c, int buf) {
                 int level, side, base, n_cols;
@@ -203,7 +204,7 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
             auto issue_s = [&](int c) {  // QR and S of chunk c
                 int level, side, base, n_cols;
                 geom(c, level, side, base, n_cols);
-                const uint32_t id_qr = tc5::instr_desc(kTcTokens, kTcRelRows, 0, 0), id_s = tc5::instr_desc(kTcTokens, n_cols, 0, 0);
+                const uint32_t id_qr = tc5::instr_desc(kTcTokens, rel_cols, 0, 0), id_s = tc5::instr_desc(kTcTokens, n_cols, 0, 0);
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
                     tc5::mma(tbase + kColQR, tc5::desc_k_major(q_u + ks * 32), tc5::desc_k_major(r_u + ks * 32), id_qr, ks > 0);
@@ -281,11 +282,13 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
             // ---- bias row -> table [offset][row]; the threads of a row share the offsets ----
             {
                 uint32_t x[16];
-                tc5::tmem_ld16(tbase + lane_base + kColQR + part * 16, x);
-                tc5::tmem_ld_wait();
+                if (part * 16 < rel_cols) {  // the same for the whole warp
+                    tc5::tmem_ld16(tbase + lane_base + kColQR + part * 16, x);
+                    tc5::tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 16; ++j) bias_s[(part * 16 + j) * kTcTokens + row] = __uint_as_float(x[j]) * scale_log2e;
-                if (part == 0) {  // offsets 64 .. 67 (k + 2 <= 66 are used)
+                    for (int j = 0; j < 16; ++j) bias_s[(part * 16 + j) * kTcTokens + row] = __uint_as_float(x[j]) * scale_log2e;
+                }
+                if (part == 0 && rel_cols > 64) {  // offsets 64 .. 67 (k + 2 <= 66 are used)
                     tc5::tmem_ld16(tbase + lane_base + kColQR + 64, x);
                     tc5::tmem_ld_wait();
 #pragma unroll
