@@ -342,6 +342,60 @@ def run_ours(args, cfg_name, cfg):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Scaling sweep (n x k grid at 262144 tokens per batch): one JSON line per point with the measured
+    step, the algorithmic FLOPs of the sparse attention and the dense full-attention FLOP / byte count
+    at the same n.  Inputs are seeded normal draws made on the device (timing only)."""
+    import torch
+    from paper_1911_04070_b200 import binding, synth
+    torch.cuda.set_device(0)
+    peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json"))) if os.path.exists(os.path.join(ROOT, "MEASURED_PEAKS.json")) else {}
+    tf_peak = float(peaks.get("bf16_tflops", 1590.0))
+    for name, cfg in synth.sweep_configs().items():
+        B, H, d, n = cfg["B"], cfg["H"], cfg["d"], cfg["n"]
+        g = binding.bpt_build_graph(n, cfg["k"], cfg["flags"], device="cuda:0")
+        gen = torch.Generator(device="cuda:0").manual_seed(cfg["seed"])
+        shape = (B, g.n_nodes, H, d)
+        q, k, v = ((torch.randn(shape, generator=gen, device="cuda:0") * cfg["std_qkv"]).bfloat16() for _ in range(3))
+        r = (torch.randn((g.n_rel, d), generator=gen, device="cuda:0") * 0.02).bfloat16()
+        d_out = torch.randn(shape, generator=gen, device="cuda:0").bfloat16()
+        ws = torch.empty(max(binding.bpt_attn_workspace_bytes(g, B, H, d, binding.BPT_BF16, True),
+                             binding.bpt_attn_workspace_bytes(g, B, H, d, binding.BPT_BF16, False), 1), dtype=torch.uint8, device="cuda:0")
+        out = torch.empty_like(q); lse = torch.empty((B, g.n_nodes, H), dtype=torch.float32, device="cuda:0")
+        dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+        d_rel = torch.empty((g.n_rel, d), dtype=torch.float32, device="cuda:0")
+
+        def step():
+            binding.bpt_attn_fwd(g, q, k, v, r, d ** -0.5, out=out, lse=lse, workspace=ws)
+            binding.bpt_attn_bwd(g, q, k, v, r, d ** -0.5, out, lse, d_out, workspace=ws, dq=dq, dk=dk, dv=dv, d_rel=d_rel)
+
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        steps = max(3, min(args.steps, 10))
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        E = g.n_edges
+        bpt_flop = 20.0 * d * B * H * E                 # algorithmic: 6d forward + 14d backward per edge and head
+        dense_flop = 14.0 * n * n * d * B * H           # full attention over the n tokens, forward + backward
+        dense_bytes = 9.0 * B * n * H * d * 2 + 8.0 * B * n * H
+        print(json.dumps({
+            "workload": name, "n": n, "k": cfg["k"], "batch": B, "edges_per_sequence": E, "ms_per_step": ms,
+            "edges_per_s": B * E / (ms * 1e-3), "tokens_per_s": B * n / (ms * 1e-3),
+            "bpt_algorithmic_tflop": bpt_flop / 1e12, "bpt_achieved_tflops": bpt_flop / (ms * 1e-3) / 1e12,
+            "dense_tflop": dense_flop / 1e12, "dense_compulsory_gb": dense_bytes / 1e9,
+            "dense_ms_at_measured_bf16_peak": dense_flop / (tf_peak * 1e12) * 1e3,
+            "dense_over_bpt_flop": dense_flop / bpt_flop,
+            "speed_vs_dense_at_peak": dense_flop / (tf_peak * 1e12) * 1e3 / ms}), flush=True)
+        del q, k, v, r, d_out, ws, out, lse, dq, dk, dv, d_rel, g
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -351,8 +405,11 @@ def main():
     ap.add_argument("--config", default="cfg4_char_lm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling of a smaller case)")
+    ap.add_argument("--sweep", action="store_true", help="run the n x k scaling sweep instead: one JSON line per point")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
+    if args.sweep:
+        return run_sweep(args)
     cfgs = all_configs()
     if args.config not in cfgs:
         raise SystemExit("unknown config %s; choose from %s" % (args.config, ", ".join(sorted(cfgs))))
