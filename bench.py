@@ -41,13 +41,13 @@ GATHER_BYTES_PER_EDGE_HEAD = {  # algorithmic bytes of the gather model, per edg
 # Which part of the gather model each kernel carries: (passes, "token" | "span" | "all" destination rows).
 KERNEL_MODEL = {
     "fwd_rows": (("fwd",), "all"), "bwd_dst": (("bwd_dst",), "all"), "bwd_src": (("bwd_src",), "all"),
-    "fwd_tile": (("fwd",), "token"), "fwd_span": (("fwd",), "span"),
+    "fwd_tile": (("fwd",), "token"), "fwd_tc5": (("fwd",), "token"), "fwd_span": (("fwd",), "span"),
     "bwd_tile": (("bwd_dst", "bwd_src"), "token"), "bwd_span": (("bwd_dst", "bwd_src"), "span"),
 }
 # DRAM bytes (read + write) per (batch entry, head) pair of one launch, from the ncu captures summarised
 # under profiles/ (taken at batch 1; every pair is an independent problem, so traffic scales with pairs).
 # An entry is dropped (traffic = null) when its kernel changes after the capture.
-NCU_DRAM_BYTES_PER_PAIR = {"fwd_tile": 41.69e6 / 8, "bwd_tile": 407.6e6 / 8}  # profiles/tile_kernels_full_cfg4_batch1.md
+NCU_DRAM_BYTES_PER_PAIR = {"fwd_tile": 41.69e6 / 8, "fwd_tc5": 41.42e6 / 8, "bwd_tile": 406.8e6 / 8}  # profiles/tile_kernels_full_cfg4_batch1.md
 
 
 def load_peaks():
