@@ -251,12 +251,14 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
         const float lse_r[2] = {lse_s[r0 + g], lse_s[r0 + g + 8]};
         const float del_r[2] = {delta_s[r0 + g], delta_s[r0 + g + 8]};
         const int w_lo = w_any ? wr.x - base : 1 << 30, w_hi = w_any ? wr.y - base : -1;
-        for (int kb = half * 32; kb <= kend; kb += 64) {
+        // every 32-key block is shared: this warp takes 16 of its keys (balanced whatever the block count)
+        for (int kb0 = 0; kb0 <= kend; kb0 += 32) {
+            const int kb = kb0 + half * 16;
             unsigned char* p_row0 = p_s + (r0 + g) * kPStride + (kb + c2) * 2;
             unsigned char* d_row0 = ds_s + (r0 + g) * kPStride + (kb + c2) * 2;
-            if (kb + 31 < w_lo || kb > w_hi) {  // nothing of these rows here: zeros for phase 2
+            if (kb + 15 < w_lo || kb > w_hi) {  // nothing of these rows here: zeros for phase 2
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < 2; ++j) {
                     *reinterpret_cast<uint32_t*>(p_row0 + j * 16) = 0u;
                     *reinterpret_cast<uint32_t*>(p_row0 + 8 * kPStride + j * 16) = 0u;
                     *reinterpret_cast<uint32_t*>(d_row0 + j * 16) = 0u;
@@ -264,28 +266,25 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 }
                 continue;
             }
-            float s[4][4], dp[4][4];
+            float s[2][4], dp[2][4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < 2; ++j) {
                 s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f;
                 dp[j][0] = dp[j][1] = dp[j][2] = dp[j][3] = 0.f;
             }
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
-#pragma unroll
-                for (int np = 0; np < 2; ++np) {
-                    uint32_t bf[4];
-                    load_b_rows(k_u, kb + np * 16, ks, lane, bf);
-                    mma_bf16(s[np * 2], qa[ks], bf[0], bf[1]);
-                    mma_bf16(s[np * 2 + 1], qa[ks], bf[2], bf[3]);
-                    load_b_rows(v_u, kb + np * 16, ks, lane, bf);
-                    mma_bf16(dp[np * 2], ga[ks], bf[0], bf[1]);
-                    mma_bf16(dp[np * 2 + 1], ga[ks], bf[2], bf[3]);
-                }
+                uint32_t bf[4];
+                load_b_rows(k_u, kb, ks, lane, bf);
+                mma_bf16(s[0], qa[ks], bf[0], bf[1]);
+                mma_bf16(s[1], qa[ks], bf[2], bf[3]);
+                load_b_rows(v_u, kb, ks, lane, bf);
+                mma_bf16(dp[0], ga[ks], bf[0], bf[1]);
+                mma_bf16(dp[1], ga[ks], bf[2], bf[3]);
             }
-            uint32_t da[2][4];
+            uint32_t da[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < 2; ++j) {
                 float pv[4], dv[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -308,19 +307,16 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 *reinterpret_cast<uint32_t*>(p_row0 + 8 * kPStride + j * 16) = p23;
                 *reinterpret_cast<uint32_t*>(d_row0 + j * 16) = d01;
                 *reinterpret_cast<uint32_t*>(d_row0 + 8 * kPStride + j * 16) = d23;
-                da[j >> 1][(j & 1) * 2] = d01;
-                da[j >> 1][(j & 1) * 2 + 1] = d23;
+                da[j * 2] = d01;
+                da[j * 2 + 1] = d23;
             }
-            // dQ += dS K
+            // dQ += dS K over these 16 keys
 #pragma unroll
-            for (int kk = 0; kk < 2; ++kk) {
-#pragma unroll
-                for (int np = 0; np < 4; ++np) {
-                    uint32_t bf[4];
-                    load_b_cols(k_u, kb + kk * 16, np, lane, bf);
-                    mma_bf16(acc_q[np * 2], da[kk], bf[0], bf[1]);
-                    mma_bf16(acc_q[np * 2 + 1], da[kk], bf[2], bf[3]);
-                }
+            for (int np = 0; np < 4; ++np) {
+                uint32_t bf[4];
+                load_b_cols(k_u, kb, np, lane, bf);
+                mma_bf16(acc_q[np * 2], da, bf[0], bf[1]);
+                mma_bf16(acc_q[np * 2 + 1], da, bf[2], bf[3]);
             }
         }
         pair_barrier(rg);  // the group's rows of the skew tile are complete
@@ -353,13 +349,15 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
         cp_async_commit();
 
         // ================= phase 2: key tiles (dk, dv partial rows) and offset tiles (d_rel partial) =================
+        // jobs: (key tile | offset tile) x (channels 0..31 | 32..63); key-tile jobs are twice as heavy, so they go first
         const int n_jt = (kend >> 4) + 1, n_ot = plan.rel_rows >> 4;
-        for (int job = w; job < n_jt + n_ot; job += kBwdThreads / 32) {
-            if (job < n_jt) {
-                const int jt = job;
-                float ak[8][4], av[8][4];
+        for (int job = w; job < 2 * (n_jt + n_ot); job += kBwdThreads / 32) {
+            const int hc = job & 1, tile16 = job >> 1;  // channel half, tile
+            if (tile16 < n_jt) {
+                const int jt = tile16;
+                float ak[4][4], av[4][4];
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) {
+                for (int nt = 0; nt < 4; ++nt) {
                     ak[nt][0] = ak[nt][1] = ak[nt][2] = ak[nt][3] = 0.f;
                     av[nt][0] = av[nt][1] = av[nt][2] = av[nt][3] = 0.f;
                 }
@@ -369,12 +367,12 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                     load_a_trans(ds_u, kPStride, ks * 16, jt * 16, lane, a_ds);
                     load_a_trans(p_u, kPStride, ks * 16, jt * 16, lane, a_p);
 #pragma unroll
-                    for (int np = 0; np < 4; ++np) {
+                    for (int np = 0; np < 2; ++np) {
                         uint32_t bf[4];
-                        load_b_cols(q_u, ks * 16, np, lane, bf);
+                        load_b_cols(q_u, ks * 16, hc * 2 + np, lane, bf);
                         mma_bf16(ak[np * 2], a_ds, bf[0], bf[1]);
                         mma_bf16(ak[np * 2 + 1], a_ds, bf[2], bf[3]);
-                        load_b_cols(g_u, ks * 16, np, lane, bf);
+                        load_b_cols(g_u, ks * 16, hc * 2 + np, lane, bf);
                         mma_bf16(av[np * 2], a_p, bf[0], bf[1]);
                         mma_bf16(av[np * 2 + 1], a_p, bf[2], bf[3]);
                     }
@@ -383,27 +381,27 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 for (int hh = 0; hh < 2; ++hh) {
                     const int m = base + jt * 16 + g + hh * 8;
                     if (m >= cr.x && m <= cr.y) {
-                        float* dst = slab_cta + (size_t)(plan.slab_row0[c] + m - cr.x) * 128 + c2;
+                        float* dst = slab_cta + (size_t)(plan.slab_row0[c] + m - cr.x) * 128 + hc * 32 + c2;
 #pragma unroll
-                        for (int nt = 0; nt < 8; ++nt) {
+                        for (int nt = 0; nt < 4; ++nt) {
                             *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ak[nt][hh * 2], ak[nt][hh * 2 + 1]);
                             *reinterpret_cast<float2*>(dst + 64 + nt * 8) = make_float2(av[nt][hh * 2], av[nt][hh * 2 + 1]);
                         }
                     }
                 }
             } else {
-                const int ot = job - n_jt;
-                float ar[8][4];
+                const int ot = tile16 - n_jt;
+                float ar[4][4];
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) { ar[nt][0] = ar[nt][1] = ar[nt][2] = ar[nt][3] = 0.f; }
+                for (int nt = 0; nt < 4; ++nt) { ar[nt][0] = ar[nt][1] = ar[nt][2] = ar[nt][3] = 0.f; }
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
                     uint32_t a[4];
                     load_a_trans(sk_u, kSkewStride, ks * 16, ot * 16, lane, a);
 #pragma unroll
-                    for (int np = 0; np < 4; ++np) {
+                    for (int np = 0; np < 2; ++np) {
                         uint32_t bf[4];
-                        load_b_cols(q_u, ks * 16, np, lane, bf);
+                        load_b_cols(q_u, ks * 16, hc * 2 + np, lane, bf);
                         mma_bf16(ar[np * 2], a, bf[0], bf[1]);
                         mma_bf16(ar[np * 2 + 1], a, bf[2], bf[3]);
                     }
@@ -411,9 +409,9 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const int o = ot * 16 + g + hh * 8;
-                    float* dst = drel_cta + ((size_t)c * plan.rel_rows + o) * 64 + c2;
+                    float* dst = drel_cta + ((size_t)c * plan.rel_rows + o) * 64 + hc * 32 + c2;
 #pragma unroll
-                    for (int nt = 0; nt < 8; ++nt)
+                    for (int nt = 0; nt < 4; ++nt)
                         *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ar[nt][hh * 2], ar[nt][hh * 2 + 1]);
                 }
             }
