@@ -198,6 +198,8 @@ def attn_fwd(g: Graph, q, k, v, r, scale):
     lse = np.zeros((B, N, H))
     for u in range(N):
         a, b = g.row_ptr[u], g.row_ptr[u + 1]
+        if a == b:                                             # a node without predecessors (only in a
+            continue                                           # length-masked graph): out = 0, lse = 0
         src, rl = g.col[a:b], g.rel[a:b]
         kk = k[:, src] + r[rl][None, :, None, :]               # [B, deg, H, d]
         s = scale * np.einsum("bhc,behc->bhe", q[:, u], kk)
@@ -230,6 +232,8 @@ def attn_bwd(g: Graph, q, k, v, r, scale, d_out, out=None):
     dr = np.zeros_like(r)
     for u in range(N):
         a, b = g.row_ptr[u], g.row_ptr[u + 1]
+        if a == b:
+            continue
         src, rl = g.col[a:b], g.rel[a:b]
         kk = k[:, src] + r[rl][None, :, None, :]
         s = scale * np.einsum("bhc,behc->bhe", q[:, u], kk)
@@ -246,4 +250,57 @@ def attn_bwd(g: Graph, q, k, v, r, scale, d_out, out=None):
         dk[:, src] += scale * np.einsum("bhe,bhc->behc", ds, q[:, u])    # src unique per row
         dv[:, src] += np.einsum("bhe,bhc->behc", p, d_out[:, u])
         np.add.at(dr, rl, scale * np.einsum("bhe,bhc->ec", ds, q[:, u]))
+    return dq, dk, dv, dr
+
+
+# ---- sequences shorter than n (placeholder tokens) ---------------------------
+#
+# The paper's tree is a perfect binary tree over n = 2^L tokens (Sec. 3.2.1) and says nothing
+# about padding.  Reading taken here: a sequence of `length` <= n real tokens occupies the first
+# `length` leaves; a node is real when it covers at least one real token.  Edges whose source or
+# destination is not real are dropped, everything else (node ids, relation ids, offsets) stays as
+# in the full graph.  Rows of nodes that are not real have no predecessors: their output and lse
+# are 0 and they receive and send no gradient.
+
+def first_token(n: int, u: int) -> int:
+    """First token covered by node id u."""
+    l, m = node_level_index(n, u)
+    return m << l
+
+
+def mask_graph(g: Graph, length: int) -> Graph:
+    """The graph restricted to the nodes that cover at least one of the first `length` tokens."""
+    if not (1 <= length <= g.n):
+        raise ValueError("length must be in [1, n]")
+    real = np.array([first_token(g.n, u) < length for u in range(g.n_nodes)])
+    dst = np.repeat(np.arange(g.n_nodes), np.diff(g.row_ptr))
+    keep = real[dst] & real[g.col]
+    deg = np.bincount(dst[keep], minlength=g.n_nodes)
+    row_ptr = np.zeros(g.n_nodes + 1, dtype=np.int32)
+    np.cumsum(deg, out=row_ptr[1:])
+    return Graph(g.n, g.k, g.flags, row_ptr, g.col[keep].copy(), g.rel[keep].copy())
+
+
+def attn_fwd_varlen(g: Graph, q, k, v, r, scale, lengths):
+    """attn_fwd with one length per batch entry (see above)."""
+    q = np.asarray(q, dtype=np.float64)
+    out = np.zeros_like(q)
+    lse = np.zeros(q.shape[:3])
+    for b, length in enumerate(lengths):
+        o, l = attn_fwd(mask_graph(g, int(length)), q[b:b + 1], np.asarray(k)[b:b + 1], np.asarray(v)[b:b + 1], r, scale)
+        out[b], lse[b] = o[0], l[0]
+    return out, lse
+
+
+def attn_bwd_varlen(g: Graph, q, k, v, r, scale, d_out, lengths, out=None):
+    """attn_bwd with one length per batch entry; dr sums over the batch."""
+    q = np.asarray(q, dtype=np.float64)
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(q), np.zeros_like(q)
+    dr = np.zeros_like(np.asarray(r, dtype=np.float64))
+    for b, length in enumerate(lengths):
+        ob = None if out is None else np.asarray(out)[b:b + 1]
+        a = attn_bwd(mask_graph(g, int(length)), q[b:b + 1], np.asarray(k)[b:b + 1], np.asarray(v)[b:b + 1], r, scale,
+                     np.asarray(d_out)[b:b + 1], out=ob)
+        dq[b], dk[b], dv[b] = a[0][0], a[1][0], a[2][0]
+        dr += a[3]
     return dq, dk, dv, dr

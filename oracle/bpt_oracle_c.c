@@ -146,6 +146,11 @@ void orc_attn_fwd(int64_t N, const int32_t* row_ptr, const int32_t* col, const i
                 const double* qu = q + (b * N + u) * rs + h * d;
                 double* ou = out + (b * N + u) * rs + h * d;
                 const int64_t a = row_ptr[u], z = row_ptr[u + 1];
+                if (a == z) { /* no predecessors (length-masked graph): out = 0, lse = 0 */
+                    for (int64_t c = 0; c < d; ++c) ou[c] = 0.0;
+                    lse[(b * N + u) * H + h] = 0.0;
+                    continue;
+                }
                 double mx = -INFINITY;
                 for (int64_t e = a; e < z; ++e) {
                     const double* kv = k + (b * N + col[e]) * rs + h * d;
@@ -203,6 +208,7 @@ void orc_attn_bwd(int64_t N, int64_t n_rel, const int32_t* row_ptr, const int32_
                 const double* qu = q + off_u;
                 const double* gu = d_out + off_u;
                 const int64_t a = row_ptr[u], z = row_ptr[u + 1];
+                if (a == z) continue;
                 double mx = -INFINITY;
                 for (int64_t e = a; e < z; ++e) {
                     const double* kv = k + (b * N + col[e]) * rs + h * d;

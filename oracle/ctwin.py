@@ -109,3 +109,49 @@ def attn_bwd(g, q, k, v, r, scale, d_out, b0=0, b1=None, out=None):
                          None if out is None else _ptr(_out),
                          _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dr))
     return dq, dk, dv, dr
+
+
+class MaskedGraph:
+    """CSR of a CGraph restricted to the nodes that cover at least one of the first `length`
+    tokens (same reading as oracle.bpt_oracle.mask_graph, written independently of it: a node id
+    is decoded level by level, its first token is index << level)."""
+
+    def __init__(self, g: CGraph, length: int):
+        n, N = g.n, g.n_nodes
+        first = np.zeros(N, dtype=np.int64)
+        base, width, level = 0, n, 0
+        while width >= 1:
+            first[base:base + width] = np.arange(width, dtype=np.int64) << level
+            base, width, level = base + width, width >> 1, level + 1
+        real = first < length
+        dst = np.repeat(np.arange(N), np.diff(g.row_ptr))
+        keep = real[dst] & real[g.col]
+        self.n, self.k, self.flags, self.L, self.n_nodes, self.n_rel = g.n, g.k, g.flags, g.L, N, g.n_rel
+        self.row_ptr = np.zeros(N + 1, dtype=np.int32)
+        np.cumsum(np.bincount(dst[keep], minlength=N), out=self.row_ptr[1:])
+        self.col = np.ascontiguousarray(g.col[keep])
+        self.rel = np.ascontiguousarray(g.rel[keep])
+        self.n_edges = int(self.col.shape[0])
+
+
+def attn_fwd_varlen(g, q, k, v, r, scale, lengths):
+    """Forward with one length per batch entry."""
+    q = _f64(q)
+    out = np.zeros_like(q)
+    lse = np.zeros(q.shape[:3])
+    for b, length in enumerate(lengths):
+        o, l = attn_fwd(MaskedGraph(g, int(length)), q, k, v, r, scale, b0=b, b1=b + 1)
+        out[b], lse[b] = o[b], l[b]
+    return out, lse
+
+
+def attn_bwd_varlen(g, q, k, v, r, scale, d_out, lengths, out=None):
+    """Backward with one length per batch entry; dr sums over the batch."""
+    q = _f64(q)
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(q), np.zeros_like(q)
+    dr = np.zeros_like(_f64(r))
+    for b, length in enumerate(lengths):
+        a = attn_bwd(MaskedGraph(g, int(length)), q, k, v, r, scale, d_out, b0=b, b1=b + 1, out=out)
+        dq[b], dk[b], dv[b] = a[0][b], a[1][b], a[2][b]
+        dr += a[3]
+    return dq, dk, dv, dr
