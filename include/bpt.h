@@ -143,6 +143,29 @@ bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt
                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The same two operations for sequences shorter than n (Sec. 3.2.1 defines the tree over a
+ * power-of-two number of tokens and is silent about other lengths; this is the library's reading).
+ * lengths: device array [B], 1 <= lengths[b] <= n (values outside are clamped).  Batch entry b has
+ * its real tokens in the first lengths[b] leaves; a node is real when it covers at least one real
+ * token.  Every edge whose source or destination is not real is dropped; node ids, relation ids and
+ * offsets stay those of the full graph, so the same bpt_graph and relation table serve all lengths.
+ * Rows of nodes that are not real: out = 0, lse = 0, dq = dk = dv = 0.
+ * The q, k, v, d_out rows of nodes that are not real never influence a result, but they must hold
+ * finite values (they may be multiplied by an exact zero weight): initialise the padding.
+ * Everything else is as for bpt_attn_fwd / bpt_attn_bwd; the forward of the backward's `out`, `lse`
+ * must have been computed with the same lengths.
+ */
+bpt_status bpt_attn_fwd_varlen(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                               const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                               const int32_t* lengths, void* out, float* lse,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+bpt_status bpt_attn_bwd_varlen(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                               const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                               const int32_t* lengths, const void* out, const float* lse, const void* d_out,
+                               void* dq, void* dk, void* dv, float* d_rel,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Backward pass for callers that must not allocate device memory (the paper has no
  * counterpart; this is a deployment convenience).
  *

@@ -19,7 +19,7 @@ BPT_F32, BPT_BF16 = 0, 1
 
 EXPORTS = ("bpt_graph_dims_query", "bpt_build_graph", "bpt_attn_workspace_bytes", "bpt_attn_fwd",
            "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end",
-           "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch")
+           "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch", "bpt_attn_fwd_varlen", "bpt_attn_bwd_varlen")
 
 
 class BptError(RuntimeError):
@@ -64,6 +64,12 @@ def load_library() -> ctypes.CDLL:
         lib.bpt_attn_bwd.restype = ctypes.c_int
         lib.bpt_attn_bwd.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
                                      vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.bpt_attn_fwd_varlen.restype = ctypes.c_int
+        lib.bpt_attn_fwd_varlen.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
+                                            vp, vp, vp, vp, sz, vp]
+        lib.bpt_attn_bwd_varlen.restype = ctypes.c_int
+        lib.bpt_attn_bwd_varlen.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
+                                            vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.bpt_static_scratch_bytes.restype = sz
         lib.bpt_static_scratch_bytes.argtypes = []
         lib.bpt_attn_bwd_static_scratch.restype = ctypes.c_int
@@ -164,8 +170,14 @@ def _check_layout(g: Graph, q, *same):
             raise ValueError("tensors must live on a CUDA device")
 
 
-def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, workspace=None):
-    """Returns (out [B,N,H,d], lse [B,N,H] fp32)."""
+def _check_lengths(lengths, q):
+    if lengths.dtype != torch.int32 or lengths.shape != (q.shape[0],) or lengths.device != q.device or not lengths.is_contiguous():
+        raise ValueError("lengths must be a contiguous int32 tensor [B] on the device of q")
+
+
+def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, workspace=None, lengths=None):
+    """Returns (out [B,N,H,d], lse [B,N,H] fp32).  With `lengths` (int32 [B] on the device) batch entry b
+    has lengths[b] real tokens; see bpt_attn_fwd_varlen in include/bpt.h."""
     lib = load_library()
     _check_layout(g, q, k, v)
     B, N, H, d = q.shape
@@ -178,15 +190,21 @@ def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, w
         need = bpt_attn_workspace_bytes(g, B, H, d, code, False)
         if workspace is None and need:
             workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
-        _check(lib.bpt_attn_fwd(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
-                                float(scale), _ptr(out), _ptr(lse), _ptr(workspace),
-                                0 if workspace is None else workspace.numel(), _stream()), "bpt_attn_fwd")
+        ws_n = 0 if workspace is None else workspace.numel()
+        if lengths is None:
+            _check(lib.bpt_attn_fwd(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
+                                    float(scale), _ptr(out), _ptr(lse), _ptr(workspace), ws_n, _stream()), "bpt_attn_fwd")
+        else:
+            _check_lengths(lengths, q)
+            _check(lib.bpt_attn_fwd_varlen(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
+                                           float(scale), _ptr(lengths), _ptr(out), _ptr(lse), _ptr(workspace), ws_n,
+                                           _stream()), "bpt_attn_fwd_varlen")
     return out, lse
 
 
 def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, workspace=None,
-                 dq=None, dk=None, dv=None, d_rel=None):
-    """Returns (dq, dk, dv [B,N,H,d], d_rel [n_rel, d] fp32)."""
+                 dq=None, dk=None, dv=None, d_rel=None, lengths=None):
+    """Returns (dq, dk, dv [B,N,H,d], d_rel [n_rel, d] fp32).  `lengths` as for bpt_attn_fwd."""
     lib = load_library()
     _check_layout(g, q, k, v, out, d_out)
     B, N, H, d = q.shape
@@ -199,10 +217,17 @@ def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, work
         need = bpt_attn_workspace_bytes(g, B, H, d, code, True)
         if workspace is None and need:
             workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
-        _check(lib.bpt_attn_bwd(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
-                                float(scale), _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq), _ptr(dk), _ptr(dv),
-                                _ptr(d_rel), _ptr(workspace), 0 if workspace is None else workspace.numel(),
-                                _stream()), "bpt_attn_bwd")
+        ws_n = 0 if workspace is None else workspace.numel()
+        if lengths is None:
+            _check(lib.bpt_attn_bwd(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
+                                    float(scale), _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq), _ptr(dk), _ptr(dv),
+                                    _ptr(d_rel), _ptr(workspace), ws_n, _stream()), "bpt_attn_bwd")
+        else:
+            _check_lengths(lengths, q)
+            _check(lib.bpt_attn_bwd_varlen(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
+                                           float(scale), _ptr(lengths), _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq),
+                                           _ptr(dk), _ptr(dv), _ptr(d_rel), _ptr(workspace), ws_n, _stream()),
+                   "bpt_attn_bwd_varlen")
     return dq, dk, dv, d_rel
 
 

@@ -21,9 +21,10 @@ extern "C" size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_
     return backward ? bwd_workspace_bytes(*g, B, H, d, dtype) : fwd_workspace_bytes(*g, B, H, d, dtype);
 }
 
-extern "C" bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
-                                   const void* q, const void* k, const void* v, const void* rel_emb, float scale,
-                                   void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+static bpt_status attn_fwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                const int32_t* lengths, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream) {
     const bpt_status s = check_problem(g, B, H, d, dtype, false);
     if (s != BPT_OK) return s;
     if (!q || !k || !v || !rel_emb || !out || !lse) return BPT_ERR_INVALID_ARG;
@@ -33,18 +34,32 @@ extern "C" bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int
     p.g = g;
     tree_params_from_dims(g->dims, &p.tree);
     p.B = B; p.H = H; p.d = d; p.dtype = dtype;
-    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths;
     p.out = out; p.lse = lse;
     p.workspace = workspace; p.workspace_bytes = workspace_bytes;
     p.stream = (cudaStream_t)cuda_stream;
     return launch_fwd(p);
 }
 
-extern "C" bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+extern "C" bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                    const void* q, const void* k, const void* v, const void* rel_emb, float scale,
-                                   const void* out, const float* lse, const void* d_out,
-                                   void* dq, void* dk, void* dv, float* d_rel,
-                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+                                   void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, out, lse, workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" bpt_status bpt_attn_fwd_varlen(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                          const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                          const int32_t* lengths, void* out, float* lse, void* workspace,
+                                          size_t workspace_bytes, void* cuda_stream) {
+    if (!lengths) return BPT_ERR_INVALID_ARG;
+    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, out, lse, workspace, workspace_bytes, cuda_stream);
+}
+
+static bpt_status attn_bwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                const int32_t* lengths, const void* out, const float* lse, const void* d_out,
+                                void* dq, void* dk, void* dv, float* d_rel,
+                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
     const bpt_status s = check_problem(g, B, H, d, dtype, true);
     if (s != BPT_OK) return s;
     if (!q || !k || !v || !rel_emb || !out || !lse || !d_out || !dq || !dk || !dv || !d_rel) return BPT_ERR_INVALID_ARG;
@@ -54,12 +69,31 @@ extern "C" bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int
     p.g = g;
     tree_params_from_dims(g->dims, &p.tree);
     p.B = B; p.H = H; p.d = d; p.dtype = dtype;
-    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths;
     p.out = const_cast<void*>(out); p.lse = const_cast<float*>(lse);
     p.d_out = d_out; p.dq = dq; p.dk = dk; p.dv = dv; p.d_rel = d_rel;
     p.workspace = workspace; p.workspace_bytes = workspace_bytes;
     p.stream = (cudaStream_t)cuda_stream;
     return launch_bwd(p);
+}
+
+extern "C" bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                   const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                   const void* out, const float* lse, const void* d_out,
+                                   void* dq, void* dk, void* dv, float* d_rel,
+                                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, out, lse, d_out, dq, dk, dv, d_rel,
+                         workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" bpt_status bpt_attn_bwd_varlen(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                          const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                          const int32_t* lengths, const void* out, const float* lse, const void* d_out,
+                                          void* dq, void* dk, void* dv, float* d_rel,
+                                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!lengths) return BPT_ERR_INVALID_ARG;
+    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, out, lse, d_out, dq, dk, dv, d_rel,
+                         workspace, workspace_bytes, cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------

@@ -52,7 +52,8 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
                const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
                const T* __restrict__ out, const float* __restrict__ lse, const T* __restrict__ d_out,
                T* __restrict__ dq, float* __restrict__ ws_p, float* __restrict__ ws_ds,
-               int N, int row0, int nrows, int H, int ngroups, int64_t e_first, int64_t E, float scale) {
+               int N, int row0, int nrows, int H, int ngroups, int64_t e_first, int64_t E, float scale,
+               const int32_t* __restrict__ lengths) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
@@ -85,6 +86,10 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
 #pragma unroll
     for (int x = 0; x < EPL; ++x) acc[x] = 0.f;
 
+    // short sequence: edges that touch a node without real tokens do not exist (their P and dS are stored as 0)
+    const int n_tok = (N + 1) / 2;
+    const int len = lengths ? min(max(lengths[b], 0), n_tok) : n_tok;
+    const bool u_real = len >= n_tok || node_first_token(n_tok, u) < len;
     const int a = row_ptr[u], z = row_ptr[u + 1];
     const size_t eoff = (size_t)b * E;
     for (int e0 = a + w * U; e0 < z; e0 += nw * U) {
@@ -94,7 +99,13 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             const int c = __shfl_sync(0xffffffffu, my_c, j), rr = __shfl_sync(0xffffffffu, my_r, j);
-            if (j < cnt) {  // uniform over the warp
+            if (j < cnt && !(u_real && (len >= n_tok || node_first_token(n_tok, c) < len))) {
+                if (sub == 0 && head_ok) {
+                    const size_t o = (eoff + (size_t)(e0 + j - e_first)) * H + head;
+                    ws_p[o] = 0.f;
+                    ws_ds[o] = 0.f;
+                }
+            } else if (j < cnt) {  // uniform over the warp
                 float kk[EPL], rv[EPL], vv[EPL];
                 M::load(k + boff + (size_t)c * rs, sub, kk);
                 M::load(r + (size_t)rr * D, sub, rv);
@@ -365,7 +376,7 @@ static bpt_status launch_bwd_rows(const AttnProblem& p) {
     const size_t smem_a = nw > 1 ? (size_t)nw * 32 * M::EPL * sizeof(float) : 0;
     bwd_dst_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem_a, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, 0, N, p.H, ngroups, 0, E, p.scale);
+        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, 0, N, p.H, ngroups, 0, E, p.scale, p.lengths);
     trace_mark(p.stream, "bwd_dst");
 
     const size_t smem_b = nw > 1 ? (size_t)nw * 32 * (2 * M::EPL) * sizeof(float) : 0;

@@ -94,7 +94,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 const __nv_bfloat16* __restrict__ out, const float* __restrict__ lse,
                 const __nv_bfloat16* __restrict__ d_out, __nv_bfloat16* __restrict__ dq,
                 int2* __restrict__ tile_range, float* __restrict__ slabs, float* __restrict__ drel_part,
-                int H, int pair0, float scale) {
+                int H, int pair0, float scale, const int32_t* __restrict__ lengths) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* q_s = smem;
     unsigned char* g_s = q_s + BwdTileSmem::q_bytes;   // d_out tile
@@ -203,6 +203,11 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
         }
     };
 
+    const int len = seq_len(lengths, b, t.n);
+    if (len < t.n) {  // short sequence: staged ranges and partial-row layout stay those of the full graph, the rows' ranges shrink
+        __syncthreads();
+        if (tid < kTileTokens) mask_row_bounds(t, t0, tid, n_left, n_right, bnd, len);
+    }
     __syncthreads();  // delta and crange are visible; the out tile in the K buffer is consumed
     stage(0);         // chunk 0 (left level 0 with the self loop) is never empty
     cp_async_commit();
@@ -613,7 +618,7 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
         bwd_tile_kernel<<<dim3(tiles, np), kBwdThreads, smem, p.stream>>>(
             t, plan, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
             (const __nv_bfloat16*)p.rel_emb, (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out,
-            (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale);
+            (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale, p.lengths);
         trace_mark(p.stream, "bwd_tile");
         const int64_t warps = (int64_t)np * N;
         bwd_gather_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, p.stream>>>(

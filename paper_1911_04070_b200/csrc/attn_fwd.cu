@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(256)
 fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col, const int32_t* __restrict__ rel,
                 const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
                 T* __restrict__ out, float* __restrict__ lse, int N, int row0, int nrows, int H, int ngroups,
-                float scale_log2e) {
+                float scale_log2e, const int32_t* __restrict__ lengths) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
@@ -43,7 +43,11 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
 #pragma unroll
     for (int c = 0; c < EPL; ++c) acc[c] = 0.f;
 
-    const int a = row_ptr[u], z = row_ptr[u + 1];
+    // short sequence: edges that touch a node without real tokens do not exist
+    const int n_tok = (N + 1) / 2;
+    const int len = lengths ? min(max(lengths[b], 0), n_tok) : n_tok;
+    const bool u_real = len >= n_tok || node_first_token(n_tok, u) < len;
+    const int a = row_ptr[u], z = u_real ? row_ptr[u + 1] : row_ptr[u];
     for (int e0 = a + w * U; e0 < z; e0 += nw * U) {
         const int cnt = min(U, z - e0);
         int my_c = 0, my_r = 0;
@@ -52,7 +56,7 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             const int c = __shfl_sync(0xffffffffu, my_c, j), rr = __shfl_sync(0xffffffffu, my_r, j);
-            if (j < cnt) {
+            if (j < cnt && (len >= n_tok || node_first_token(n_tok, c) < len)) {
                 float kk[EPL], rv[EPL];
                 M::load(k + boff + (size_t)c * rs, sub, kk);
                 M::load(r + (size_t)rr * D, sub, rv);
@@ -73,13 +77,14 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
             s[j] = M::head_sum(s[j]);
             m_new = fmaxf(m_new, s[j]);
         }
-        const float corr = fast_exp2(m - m_new);
+        const float m_ref = m_new == -INFINITY ? 0.f : m_new;  // nothing seen so far (only skipped edges): keep the empty state
+        const float corr = fast_exp2(m - m_ref);
         l *= corr;
 #pragma unroll
         for (int x = 0; x < EPL; ++x) acc[x] *= corr;
 #pragma unroll
         for (int j = 0; j < U; ++j) {
-            const float p = fast_exp2(s[j] - m_new);
+            const float p = fast_exp2(s[j] - m_ref);
             l += p;
 #pragma unroll
             for (int x = 0; x < EPL; ++x) acc[x] = fmaf(p, vv[j][x], acc[x]);
@@ -99,6 +104,7 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
         if (w != 0) return;
         float mt = -INFINITY;
         for (int j = 0; j < nw; ++j) mt = fmaxf(mt, sm_m[j * 32 + lane]);
+        if (mt == -INFINITY) mt = 0.f;  // a row without edges: every warp state is empty
         l = 0.f;
 #pragma unroll
         for (int x = 0; x < EPL; ++x) acc[x] = 0.f;
@@ -115,7 +121,7 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
     for (int x = 0; x < EPL; ++x) acc[x] *= inv;
     if (head_ok) {
         M::store(out + boff + (size_t)u * rs, sub, acc);
-        if (sub == 0) lse[((size_t)b * N + u) * H + head] = (m + log2f(l)) * kLn2;
+        if (sub == 0) lse[((size_t)b * N + u) * H + head] = l > 0.f ? (m + log2f(l)) * kLn2 : 0.f;
     }
 }
 
@@ -137,7 +143,7 @@ static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows) {
     const size_t smem = nw > 1 ? (size_t)nw * 32 * (2 + M::EPL) * sizeof(float) : 0;
     fwd_rows_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e);
+        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e, p.lengths);
     trace_mark(p.stream, "fwd_rows");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }
@@ -171,7 +177,7 @@ static bool want_tc5(int k) {
 bpt_status launch_fwd(const AttnProblem& p) {
     if (tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16)) {  // token rows and span rows on the tensor cores
         int* status = reinterpret_cast<int*>(static_cast<char*>(p.workspace) + span_ws_bytes(p.tree, p.B, p.H));
-        const bpt_status s = (want_tc5(p.tree.k) && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, status) : launch_fwd_tile(p);
+        const bpt_status s = (want_tc5(p.tree.k) && !p.lengths && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, status) : launch_fwd_tile(p);
         return s != BPT_OK ? s : launch_fwd_span(p);
     }
     const int row0 = 0, nrows = p.g->dims.n_nodes;

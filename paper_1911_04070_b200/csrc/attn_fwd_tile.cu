@@ -43,7 +43,8 @@ __global__ void __launch_bounds__(128)
 fwd_tile_kernel(TreeParams t, int n_left, int n_right,
                 const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                 const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
-                __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int H, float scale_log2e) {
+                __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int H, float scale_log2e,
+                const int32_t* __restrict__ lengths) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* q_s = smem;
     unsigned char* k_s = q_s + FwdTileSmem::q_bytes;
@@ -79,6 +80,11 @@ fwd_tile_kernel(TreeParams t, int n_left, int n_right,
         const int2 a = rows_union(bnd + c * kTileTokens, 0, 32, lane);
         const int2 bb = rows_union(bnd + c * kTileTokens, 32, 32, lane);
         if (lane == 0) crange[c] = make_int2(min(a.x, bb.x), max(a.y, bb.y));
+    }
+    const int len = seq_len(lengths, b, t.n);
+    if (len < t.n) {  // short sequence: the staged ranges stay those of the full graph, the rows' ranges shrink
+        __syncthreads();
+        if (tid < kTileTokens) mask_row_bounds(t, t0, tid, n_left, n_right, bnd, len);
     }
 
     const int r0 = w * 16;
@@ -254,7 +260,7 @@ fwd_tile_kernel(TreeParams t, int n_left, int n_right,
     for (int hh = 0; hh < 2; ++hh) {
         l_run[hh] += __shfl_xor_sync(0xffffffffu, l_run[hh], 1);
         l_run[hh] += __shfl_xor_sync(0xffffffffu, l_run[hh], 2);
-        inv[hh] = 1.f / l_run[hh];
+        inv[hh] = t0 + r0 + g + hh * 8 < len ? 1.f / l_run[hh] : 0.f;  // a placeholder token's row is zero
     }
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt) {
@@ -264,7 +270,7 @@ fwd_tile_kernel(TreeParams t, int n_left, int n_right,
     if ((lane & 3) == 0) {
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh)
-            lse[((size_t)b * N + t0 + r0 + g + hh * 8) * H + h] = (m_run[hh] + log2f(l_run[hh])) * kLn2;
+            lse[((size_t)b * N + t0 + r0 + g + hh * 8) * H + h] = inv[hh] > 0.f ? (m_run[hh] + log2f(l_run[hh])) * kLn2 : 0.f;
     }
     __syncwarp();
     for (int idx = lane; idx < 16 * 8; idx += 32) {
@@ -288,7 +294,7 @@ bpt_status launch_fwd_tile(const AttnProblem& p) {
     fwd_tile_kernel<<<grid, 128, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q,
                                                    (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
                                                    (const __nv_bfloat16*)p.rel_emb, (__nv_bfloat16*)p.out, p.lse, p.H,
-                                                   p.scale * kLog2e);
+                                                   p.scale * kLog2e, p.lengths);
     trace_mark(p.stream, "fwd_tile");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }

@@ -33,8 +33,8 @@ struct SpanRow {
     int level;
 };
 
-// Row r of the tile's span matrix.
-__device__ __forceinline__ SpanRow span_row(const TreeParams& t, int t0, int r) {
+// Row r of the tile's span matrix; `len` = real tokens of the sequence (a span attends only those).
+__device__ __forceinline__ SpanRow span_row(const TreeParams& t, int t0, int r, int len) {
     SpanRow s;
     s.node = -1; s.lo = 1; s.hi = 0; s.level = 1;
     if (r < kTileTokens - 1) {
@@ -56,6 +56,8 @@ __device__ __forceinline__ SpanRow span_row(const TreeParams& t, int t0, int r) 
             s.hi = kTileTokens - 1;
         }
     }
+    s.hi = min(s.hi, len - 1 - t0);
+    if (s.lo > s.hi) { s.lo = 1; s.hi = 0; }  // no real token of this tile under the span
     return s;
 }
 
@@ -73,7 +75,7 @@ __global__ void __launch_bounds__(kSpanThreads)
 fwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                 const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
                 __nv_bfloat16* __restrict__ out, float* __restrict__ lse, float* __restrict__ ext_part,
-                int H, int n_ext, float scale_log2e) {
+                int H, int n_ext, float scale_log2e, const int32_t* __restrict__ lengths) {
     __shared__ __align__(128) unsigned char qs_s[kSpanRows * 128];
     __shared__ __align__(128) unsigned char k_s[kTileTokens * 128];
     __shared__ __align__(128) unsigned char v_s[kTileTokens * 128];
@@ -87,7 +89,7 @@ fwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
     const uint32_t qs_u = smem_u32(qs_s), k_u = smem_u32(k_s), v_u = smem_u32(v_s);
 
     if (tid < kSpanRows) {
-        const SpanRow s = span_row(t, t0, tid);
+        const SpanRow s = span_row(t, t0, tid, seq_len(lengths, b, t.n));
         meta.node[tid] = s.node; meta.lo[tid] = s.lo; meta.hi[tid] = s.hi; meta.level[tid] = s.level;
     }
     __syncthreads();
@@ -208,8 +210,8 @@ fwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
 #pragma unroll
             for (int nt = 0; nt < 8; ++nt)
                 *reinterpret_cast<uint32_t*>(qs_s + tile_off(row, nt) + c2 * 2) = pack_bf16(o[nt][hh * 2] * inv, o[nt][hh * 2 + 1] * inv);
-            if ((lane & 3) == 0 && meta.node[row] >= 0)
-                lse[((size_t)b * N + meta.node[row]) * H + h] = (mx[hh] + log2f(l_run[hh])) * kLn2;
+            if ((lane & 3) == 0 && meta.node[row] >= 0)  // a span without real tokens: out = 0, lse = 0
+                lse[((size_t)b * N + meta.node[row]) * H + h] = l_run[hh] > 0.f ? (mx[hh] + log2f(l_run[hh])) * kLn2 : 0.f;
         }
         __syncwarp();
         for (int idx = lane; idx < 16 * 8; idx += 32) {
@@ -257,16 +259,16 @@ fwd_span_merge_kernel(TreeParams t, const float* __restrict__ ext_part, __nv_bfl
 #pragma unroll 4
     for (int x = 0; x < nT; ++x) {
         const float* p = base + (size_t)x * stride;
-        const float f = fast_exp2(p[0] - mx);
+        const float f = mx == -INFINITY ? 0.f : fast_exp2(p[0] - mx);
         const float2 a = *reinterpret_cast<const float2*>(p + 2 + lane * 2);
         l = fmaf(p[1], f, l);
         a0 = fmaf(a.x, f, a0);
         a1 = fmaf(a.y, f, a1);
     }
-    const float inv = 1.f / l;
+    const float inv = l > 0.f ? 1.f / l : 0.f;  // l = 0: a span without real tokens
     const size_t rs = (size_t)H * 64;
     *reinterpret_cast<uint32_t*>(out + ((size_t)b * (2 * t.n - 1) + node) * rs + (size_t)h * 64 + lane * 2) = pack_bf16(a0 * inv, a1 * inv);
-    if (lane == 0) lse[((size_t)b * (2 * t.n - 1) + node) * H + h] = (mx + log2f(l)) * kLn2;
+    if (lane == 0) lse[((size_t)b * (2 * t.n - 1) + node) * H + h] = l > 0.f ? (mx + log2f(l)) * kLn2 : 0.f;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -278,7 +280,7 @@ bwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
                 const __nv_bfloat16* __restrict__ out, const float* __restrict__ lse,
                 const __nv_bfloat16* __restrict__ d_out, __nv_bfloat16* __restrict__ dq,
                 float* __restrict__ ext_dq, float* __restrict__ aff_slab,
-                int H, int pair0, int n_ext, float scale) {
+                int H, int pair0, int n_ext, float scale, const int32_t* __restrict__ lengths) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* qs_s = smem;
     unsigned char* gs_s = qs_s + kSpanRows * 128;
@@ -300,7 +302,7 @@ bwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
     unsigned char* o_s = p_s;  // the spans' forward outputs, only until the row terms are known (80 x 128 <= 80 x 144)
 
     if (tid < kSpanRows) {
-        const SpanRow s = span_row(t, t0, tid);
+        const SpanRow s = span_row(t, t0, tid, seq_len(lengths, b, t.n));
         meta.node[tid] = s.node; meta.lo[tid] = s.lo; meta.hi[tid] = s.hi; meta.level[tid] = s.level;
         meta.lse2[tid] = s.node >= 0 ? lse[((size_t)b * N + s.node) * H + h] * kLog2e : 0.f;
     }
@@ -549,7 +551,7 @@ bpt_status launch_fwd_span(const AttnProblem& p) {
     float* ext = (float*)p.workspace;
     fwd_span_kernel<<<dim3(tiles, p.H, p.B), kSpanThreads, 0, p.stream>>>(
         t, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v, (const __nv_bfloat16*)p.rel_emb,
-        (__nv_bfloat16*)p.out, p.lse, ext, p.H, n_ext, p.scale * kLog2e);
+        (__nv_bfloat16*)p.out, p.lse, ext, p.H, n_ext, p.scale * kLog2e, p.lengths);
     trace_mark(p.stream, "fwd_span");
     if (n_ext > 0) {
         const int64_t warps = (int64_t)p.B * p.H * (tiles - 1);
@@ -574,7 +576,7 @@ bpt_status launch_bwd_span(const AttnProblem& p, int pair0, int n_pairs, float* 
     bwd_span_kernel<<<dim3(tiles, n_pairs), kSpanThreads, kBwdSpanSmem, p.stream>>>(
         t, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v, (const __nv_bfloat16*)p.rel_emb,
         (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out, (__nv_bfloat16*)p.dq, ext_dq, aff_slab,
-        p.H, pair0, n_ext, p.scale);
+        p.H, pair0, n_ext, p.scale, p.lengths);
     trace_mark(p.stream, "bwd_span");
     if (n_ext > 0) {
         const int64_t warps = (int64_t)n_pairs * (tiles - 1);

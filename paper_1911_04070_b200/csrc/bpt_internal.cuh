@@ -19,6 +19,7 @@ struct AttnProblem {
     int B, H, d;
     bpt_dtype dtype;
     const void *q, *k, *v, *rel_emb;
+    const int32_t* lengths;  // [B] real tokens per batch entry, or nullptr: all n (see bpt_attn_fwd_varlen)
     float scale;
     // forward outputs / backward inputs
     void* out;

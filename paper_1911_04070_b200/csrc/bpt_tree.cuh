@@ -28,6 +28,13 @@ BPT_HD int node_level(int n, int u) {
     return l;
 }
 
+// first token covered by node id u
+BPT_HD int node_first_token(int n, int u) {
+    int l = 0, base = 0, width = n;
+    while (u >= base + width) { base += width; width >>= 1; ++l; }
+    return (u - base) << l;
+}
+
 BPT_HD int rel_left(const TreeParams& t, int j, int o) { return 1 + j * (t.k + 1) + o; }
 BPT_HD int rel_right(const TreeParams& t, int j, int o) { return 1 + (t.L + j) * (t.k + 1) + o; }
 BPT_HD int rel_anc(const TreeParams& t, int j) { return 1 + 2 * t.L * (t.k + 1) + (j - 1); }

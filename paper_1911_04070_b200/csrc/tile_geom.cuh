@@ -47,6 +47,30 @@ __device__ __forceinline__ void fill_row_bounds(const TreeParams& t, int t0, int
     }
 }
 
+// Sequences shorter than n: the first `len` tokens are real, a node is real when it covers a real
+// token, i.e. node (level, m) with m <= (len - 1) >> level; edges that touch other nodes do not exist.
+__device__ __forceinline__ int seq_len(const int32_t* lengths, int b, int n) {
+    return lengths ? min(max(lengths[b], 0), n) : n;
+}
+
+// Applies a length to the row ranges fill_row_bounds wrote for token t0 + r: a placeholder token
+// attends nothing; a real token's right-side ranges end at the last real node of the level (left-side
+// nodes lie before the token and are real).  Empty ranges keep the encoding of fill_row_bounds.
+template <int TILE = kTileTokens>
+__device__ __forceinline__ void mask_row_bounds(const TreeParams& t, int t0, int r, int n_left, int n_right, int2* bnd, int len) {
+    if (len >= t.n) return;
+    const bool real = t0 + r < len;
+    for (int c = 0; c < n_left; ++c)
+        if (!real) bnd[c * TILE + r] = make_int2(0, -1);
+    for (int c = 0; c < n_right; ++c) {
+        const int n_l = t.n >> c;
+        int2 v = bnd[(n_left + c) * TILE + r];
+        if (real && v.x <= v.y) v.y = min(v.y, (len - 1) >> c);
+        if (!real || v.x > v.y) v = make_int2(n_l, n_l - 1);
+        bnd[(n_left + c) * TILE + r] = v;
+    }
+}
+
 // Union of the non-empty ranges of rows [r0, r0 + cnt) of one chunk (lanes 0..cnt-1 each
 // look at one row; cnt <= 32).  Returns (lo, hi) with lo > hi when all rows are empty.
 __device__ __forceinline__ int2 rows_union(const int2* bnd_chunk, int r0, int cnt, int lane) {
