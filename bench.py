@@ -396,6 +396,49 @@ def run_sweep(args):
         torch.cuda.empty_cache()
 
 
+def run_model(args):
+    """Whole-model figure in the setting of the paper's Sec. 4.4 (6 layers, d = 512, d_ff = 2048, 8 heads,
+    8192 tokens per batch, bf16): tokens/s of a forward pass (inference) and of a forward + backward pass
+    through BPTEncoder, for a few sequence lengths and k.  One JSON line per point."""
+    import torch
+    from paper_1911_04070_b200 import layer
+    torch.cuda.set_device(0)
+    torch.manual_seed(0)
+    for n in (512, 2048, 8192):
+        for k in (4, 16, 64):
+            B = 8192 // n
+            enc = layer.BPTEncoder(n, k, 512, 8, 2048, 6, left_only=True, device="cuda:0").to("cuda:0", torch.bfloat16)
+            x = torch.randn(B, n, 512, device="cuda:0", dtype=torch.bfloat16, requires_grad=True)
+
+            def fwd():
+                with torch.no_grad():
+                    enc(x)
+
+            def train():
+                enc.zero_grad(set_to_none=True)
+                enc(x).float().square().mean().backward()
+
+            res = {}
+            for name, fn in (("forward", fwd), ("forward_backward", train)):
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                steps = max(3, min(args.steps, 10))
+                e0.record()
+                for _ in range(steps):
+                    fn()
+                e1.record()
+                torch.cuda.synchronize()
+                res[name] = e0.elapsed_time(e1) / steps
+            print(json.dumps({"workload": "6-layer BPT stack, d=512, d_ff=2048, 8 heads, left-only, 8192 tokens per batch, bf16",
+                              "n": n, "k": k, "batch": B, "forward_ms": res["forward"], "forward_tokens_per_s": 8192 / (res["forward"] * 1e-3),
+                              "forward_backward_ms": res["forward_backward"],
+                              "forward_backward_tokens_per_s": 8192 / (res["forward_backward"] * 1e-3)}), flush=True)
+            del enc, x
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -406,10 +449,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling of a smaller case)")
     ap.add_argument("--sweep", action="store_true", help="run the n x k scaling sweep instead: one JSON line per point")
+    ap.add_argument("--model", action="store_true", help="time a 6-layer BPT stack (Sec. 4.4 setting) instead: one JSON line per point")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.sweep:
         return run_sweep(args)
+    if args.model:
+        return run_model(args)
     cfgs = all_configs()
     if args.config not in cfgs:
         raise SystemExit("unknown config %s; choose from %s" % (args.config, ", ".join(sorted(cfgs))))

@@ -1,0 +1,96 @@
+"""BP-Transformer layers on top of the graph self-attention library (arXiv 1911.04070, Sec. 3.3,
+Algorithm 2): PyTorch modules whose attention runs in libbpt.so.
+
+Only the graph self-attention is this package's own code; the projections, the feed-forward block
+and the layer normalisation are plain PyTorch operators around it, so that the operator can be
+dropped into a model and trained.  Nothing here falls back to another attention implementation.
+"""
+from __future__ import annotations
+
+import math
+
+import torch
+from torch import nn
+
+from . import binding
+
+
+class _GraphSelfAttention(torch.autograd.Function):
+    """out = GSA(q, k, v, rel_emb) over the BPT graph; backward through bpt_attn_bwd."""
+
+    @staticmethod
+    def forward(ctx, q, k, v, rel_emb, g, scale, lengths):
+        q, k, v, rel_emb = q.contiguous(), k.contiguous(), v.contiguous(), rel_emb.contiguous()
+        out, lse = binding.bpt_attn_fwd(g, q, k, v, rel_emb, scale, lengths=lengths)
+        ctx.save_for_backward(q, k, v, rel_emb, out, lse)
+        ctx.g, ctx.scale, ctx.lengths = g, scale, lengths
+        return out
+
+    @staticmethod
+    def backward(ctx, d_out):
+        q, k, v, rel_emb, out, lse = ctx.saved_tensors
+        dq, dk, dv, d_rel = binding.bpt_attn_bwd(ctx.g, q, k, v, rel_emb, ctx.scale, out, lse, d_out.contiguous(),
+                                                 lengths=ctx.lengths)
+        return dq, dk, dv, d_rel.to(rel_emb.dtype), None, None, None
+
+
+def graph_self_attention(g: binding.Graph, q, k, v, rel_emb, scale=None, lengths=None):
+    """Differentiable graph self-attention with tree relative positions (Sec. 3.1, 3.4).
+
+    q, k, v: [B, 2n-1, H, d] (float32 or bfloat16, on the graph's device); rel_emb: [n_rel, d], shared
+    by the heads; lengths: optional int32 [B].  Returns [B, 2n-1, H, d]."""
+    scale = 1.0 / math.sqrt(q.shape[-1]) if scale is None else float(scale)
+    return _GraphSelfAttention.apply(q, k, v, rel_emb, g, scale, lengths)
+
+
+class BPTLayer(nn.Module):
+    """One layer of Algorithm 2:  Z = norm(H + GSA(H)),  H' = norm(Z + FFN(Z)).
+
+    H holds the states of all 2n-1 nodes.  The relation embeddings are a parameter of the layer
+    (Sec. 3.4: not shared between layers, shared between the heads)."""
+
+    def __init__(self, g: binding.Graph, d_model: int, n_heads: int, d_ff: int, rel_std: float = 0.02):
+        super().__init__()
+        if d_model % n_heads:
+            raise ValueError("d_model must be a multiple of n_heads")
+        self.g, self.h, self.dh = g, n_heads, d_model // n_heads
+        self.wq, self.wk, self.wv, self.wo = (nn.Linear(d_model, d_model, bias=False) for _ in range(4))
+        self.rel_emb = nn.Parameter(torch.randn(g.n_rel, self.dh) * rel_std)
+        self.norm1, self.norm2 = nn.LayerNorm(d_model), nn.LayerNorm(d_model)
+        self.ff1, self.ff2 = nn.Linear(d_model, d_ff), nn.Linear(d_ff, d_model)
+
+    def forward(self, h, lengths=None):
+        B, N, D = h.shape
+        split = lambda x: x.view(B, N, self.h, self.dh)
+        a = graph_self_attention(self.g, split(self.wq(h)), split(self.wk(h)), split(self.wv(h)),
+                                 self.rel_emb.to(h.dtype), lengths=lengths)
+        z = self.norm1(h + self.wo(a.reshape(B, N, D)))
+        return self.norm2(z + self.ff2(torch.relu(self.ff1(z))))
+
+
+class BPTEncoder(nn.Module):
+    """A stack of BPT layers over one sequence length n (a power of two).
+
+    Token nodes start from the given token states, span nodes from zero, and all nodes are updated
+    together in every layer (Sec. 3.3).  `readout`: "tokens" returns the token states [B, n, D]
+    (language modelling, translation), "root" the root node's state [B, D] (classification)."""
+
+    def __init__(self, n: int, k: int, d_model: int, n_heads: int, d_ff: int, n_layers: int, left_only: bool = False,
+                 device="cuda"):
+        super().__init__()
+        self.n = n
+        self.g = binding.bpt_build_graph(n, k, binding.BPT_LEFT_ONLY if left_only else 0, device=device)
+        self.layers = nn.ModuleList(BPTLayer(self.g, d_model, n_heads, d_ff) for _ in range(n_layers))
+
+    def forward(self, tokens, lengths=None, readout: str = "tokens"):
+        B, n, D = tokens.shape
+        if n != self.n:
+            raise ValueError("expected %d token states per sequence, got %d" % (self.n, n))
+        h = torch.cat([tokens, tokens.new_zeros(B, n - 1, D)], dim=1)
+        for layer in self.layers:
+            h = layer(h, lengths)
+        if readout == "tokens":
+            return h[:, :n]
+        if readout == "root":
+            return h[:, -1]
+        raise ValueError("readout must be 'tokens' or 'root'")
