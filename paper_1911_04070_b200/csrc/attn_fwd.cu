@@ -177,7 +177,7 @@ static bool want_tc5(int k) {
 bpt_status launch_fwd(const AttnProblem& p) {
     if (tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16)) {  // token rows and span rows on the tensor cores
         int* status = reinterpret_cast<int*>(static_cast<char*>(p.workspace) + span_ws_bytes(p.tree, p.B, p.H));
-        const bpt_status s = (want_tc5(p.tree.k) && !p.lengths && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, status) : launch_fwd_tile(p);
+        const bpt_status s = (want_tc5(p.tree.k) && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, status) : launch_fwd_tile(p);
         return s != BPT_OK ? s : launch_fwd_span(p);
     }
     const int row0 = 0, nrows = p.g->dims.n_nodes;

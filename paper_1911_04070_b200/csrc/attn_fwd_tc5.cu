@@ -84,7 +84,7 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
                const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
                __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int* __restrict__ status,
-               int H, float scale_log2e, const __grid_constant__ CUtensorMap tm_k,
+               int H, float scale_log2e, const int32_t* __restrict__ lengths, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_r) {
     extern __shared__ unsigned char smem_raw[];
     // the swizzle pattern is a function of the address bits, so the tiles must start 1024-aligned
@@ -157,6 +157,13 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
         if (lane == 0) crange[c] = u;
     }
     __syncthreads();
+    {   // short sequence: the staged ranges stay those of the full graph, the rows' ranges shrink
+        const int len = seq_len(lengths, b, t.n);
+        if (len < t.n) {
+            if (tid < kTcTokens) mask_row_bounds<kTcTokens>(t, t0, tid, n_left, n_right, bnd_abs, len);
+            __syncthreads();
+        }
+    }
     for (int idx = tid; idx < chunks * kTcTokens; idx += kTcThreads) {
         const int2 a = bnd_abs[idx];
         const int base = crange[idx / kTcTokens].x;
@@ -401,7 +408,7 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
             for (int x = 0; x < 4; ++x) pk[x] = pack_bf16(o[ch * 8 + 2 * x] * inv, o[ch * 8 + 2 * x + 1] * inv);
             *reinterpret_cast<uint4*>(q_s + tile_off(row, part * (kChan / 8) + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
-        if (part == 0) lse[((size_t)b * N_nodes + t0 + row) * H + h] = (m_run + log2f(l_all)) * kLn2;
+        if (part == 0) lse[((size_t)b * N_nodes + t0 + row) * H + h] = l_all > 0.f ? (m_run + log2f(l_all)) * kLn2 : 0.f;
     }
 
     // ---- epilogue: coalesced stores of the output tile; tensor memory back ----
@@ -484,7 +491,7 @@ bpt_status launch_fwd_tc5(const AttnProblem& p, int* status) {
     fwd_tc5_kernel<<<grid, kTcThreads, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q,
                                                          (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
                                                          (const __nv_bfloat16*)p.rel_emb, (__nv_bfloat16*)p.out, p.lse,
-                                                         status, p.H, p.scale * kLog2e, tm_k, tm_v, tm_r);
+                                                         status, p.H, p.scale * kLog2e, p.lengths, tm_k, tm_v, tm_r);
     trace_mark(p.stream, "fwd_tc5");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }

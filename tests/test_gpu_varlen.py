@@ -67,7 +67,7 @@ CASES = [
     (64, 4, 0, 2, 64, True, [64, 37, 1]),                 # one tile
     (256, 4, 0, 3, 64, True, [256, 100, 65, 64]),         # tile boundaries
     (512, 16, 1, 2, 64, True, [300, 511]),
-    (1024, 64, 0, 1, 64, True, [1000, 129]),              # k = 64: the length path uses the warp-level forward
+    (1024, 64, 0, 1, 64, True, [1000, 129]),              # k = 64: tensor-memory forward
     (2048, 8, 2, 2, 64, True, [1500, 2048, 7]),
     (4096, 3, 0, 1, 64, True, [4000, 2049]),              # outer ancestors with and without real tokens
 ]
