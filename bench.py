@@ -245,16 +245,35 @@ def run_ours(args, cfg_name, cfg):
     if rank == 0:
         sampler.start()
     cap = min(args.steps * 16 + 8, 4000)
-    binding.bpt_trace_begin(cap)
+    # L2 (126 MB): a workload whose tensors exceed it evicts itself between steps; a smaller one gets a
+    # 256 MB write between the timed steps, which are then timed one by one
+    in_bytes = sum(v.numel() * v.element_size() for v in t.values()) + out.numel() * out.element_size()
+    flush = in_bytes < 192 * 1024 * 1024
+    scrub = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev) if flush else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
-    marks = binding.bpt_trace_end(cap)
+    if not flush:
+        binding.bpt_trace_begin(cap)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+        ms_sum = e0.elapsed_time(e1)
+        marks = binding.bpt_trace_end(cap)
+    else:
+        ms_sum, marks = 0.0, []
+        for _ in range(args.steps):
+            scrub.zero_()
+            binding.bpt_trace_begin(16)
+            e0.record()
+            step()
+            e1.record()
+            torch.cuda.synchronize()
+            ms_sum += e0.elapsed_time(e1)
+            marks += binding.bpt_trace_end(16)
+        barrier()
+    ms_total = max_over_ranks(ms_sum)
     clocks = sampler.stop() if rank == 0 else None
     ms_step = ms_total / args.steps
     value = world * B * E / (ms_step * 1e-3)
@@ -324,7 +343,8 @@ def run_ours(args, cfg_name, cfg):
         "dtype": "bf16" if cfg["bf16"] else "f32", "data": "synthetic",
         "config": {"workload": cfg_name, "n": cfg["n"], "k": cfg["k"], "left_only": bool(cfg["flags"] & 1),
                    "batch_per_gpu": B, "heads": H, "d_head": d, "edges_per_sequence": E,
-                   "pass": "fwd+bwd" if do_bwd else "fwd", "l2": "inputs larger than L2", "parallelism": "batch shards x%d" % world},
+                   "pass": "fwd+bwd" if do_bwd else "fwd",
+                   "l2": "flushed by a 256 MB write between timed steps" if flush else "inputs larger than L2", "parallelism": "batch shards x%d" % world},
         "edge_heads_per_s": value * H, "tokens_per_s": world * B * cfg["n"] / (ms_step * 1e-3),
         "hbm_roofline_frac_step": step_roof_ms / ms_step, "hbm_roofline_ms_step": step_roof_ms,
         "compulsory_hbm_ms_step": compulsory_ms, "compulsory_hbm_frac_step": compulsory_ms / ms_step,
