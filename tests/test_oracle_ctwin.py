@@ -14,7 +14,7 @@ def test_graph(n, k, flags):
         assert np.array_equal(getattr(g, name), getattr(c, name)), name
 
 
-def test_survey_scale_edge_counts():
+def test_mid_size_edge_counts():
     # E = E_ctx + n + n log2 n; E_aff and E_self are fixed by Sec. 3.2.2, so this pins E_ctx of the twin
     # against the NumPy enumeration on a mid-sized case and the twin's own count routine elsewhere.
     c = ctwin.CGraph(2048, 8, 0)
