@@ -304,3 +304,103 @@ def attn_bwd_varlen(g: Graph, q, k, v, r, scale, d_out, lengths, out=None):
         dq[b], dk[b], dv[b] = a[0][0], a[1][0], a[2][0]
         dr += a[3]
     return dq, dk, dv, dr
+
+
+# ---- attention dropout (App. A.1 lists an attention dropout rate p_a for every experiment) --------
+#
+# The paper does not say how its masks are drawn.  Here every edge weight of every (batch entry,
+# head) is kept with probability 1 - p and divided by 1 - p (inverted dropout, applied after the
+# softmax, before the product with V), and the mask is a pure function of (seed, batch entry, head,
+# destination node, source node) so that the backward pass and another implementation can rebuild
+# it: Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as
+# 1, 2, 3", SC'11), key = (seed & 0xffffffff, seed >> 32), counter = (destination node, source node,
+# batch entry * H + head, PHILOX_TAG), first output word u; the edge is kept iff u >= floor(p * 2^32).
+
+PHILOX_M0, PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+PHILOX_W0, PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+PHILOX_TAG = 0x42505431
+
+
+def philox4x32_10(c0, c1, c2, c3, k0, k1):
+    """Philox4x32-10 on arrays (or scalars) of 32-bit words; returns the four output words."""
+    c0, c1, c2, c3 = (np.asarray(a, dtype=np.uint64) & np.uint64(0xFFFFFFFF) for a in (c0, c1, c2, c3))
+    k0, k1 = np.uint64(k0 & 0xFFFFFFFF), np.uint64(k1 & 0xFFFFFFFF)
+    mask = np.uint64(0xFFFFFFFF)
+    for _ in range(10):
+        p0 = np.uint64(PHILOX_M0) * c0          # 64-bit products of 32-bit words
+        p1 = np.uint64(PHILOX_M1) * c2
+        hi0, lo0, hi1, lo1 = p0 >> np.uint64(32), p0 & mask, p1 >> np.uint64(32), p1 & mask
+        c0, c1, c2, c3 = hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0
+        k0 = (k0 + np.uint64(PHILOX_W0)) & mask
+        k1 = (k1 + np.uint64(PHILOX_W1)) & mask
+    return c0, c1, c2, c3
+
+
+def dropout_keep(seed: int, p: float, b: int, h: int, H: int, dst, src):
+    """Boolean keep mask of the edges src[i] -> dst[i] for batch entry b and head h."""
+    thr = np.uint64(min(int(np.floor(float(p) * 4294967296.0)), 0xFFFFFFFF))
+    u = philox4x32_10(dst, src, np.full(np.shape(src), b * H + h), np.full(np.shape(src), PHILOX_TAG),
+                      seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)[0]
+    return u >= thr
+
+
+def attn_fwd_dropout(g: Graph, q, k, v, r, scale, p_drop, seed):
+    """attn_fwd with attention dropout: out_u = sum_e keep_e / (1 - p) P_e v_v; lse is that of the softmax."""
+    q, k, v, r = (np.asarray(a, dtype=np.float64) for a in (q, k, v, r))
+    B, N, H, d = q.shape
+    out = np.zeros_like(q)
+    lse = np.zeros((B, N, H))
+    for u in range(N):
+        a, b_ = g.row_ptr[u], g.row_ptr[u + 1]
+        if a == b_:
+            continue
+        src, rl = g.col[a:b_], g.rel[a:b_]
+        kk = k[:, src] + r[rl][None, :, None, :]
+        s = scale * np.einsum("bhc,behc->bhe", q[:, u], kk)
+        mx = s.max(axis=2, keepdims=True)
+        pr = np.exp(s - mx)
+        z = pr.sum(axis=2, keepdims=True)
+        pr = pr / z
+        lse[:, u] = (mx + np.log(z))[:, :, 0]
+        for b in range(B):
+            for h in range(H):
+                keep = dropout_keep(seed, p_drop, b, h, H, np.full(src.shape, u), src)
+                w = pr[b, h] * keep / (1.0 - p_drop)
+                out[b, u, h] = w @ v[b, src, h]
+    return out, lse
+
+
+def attn_bwd_dropout(g: Graph, q, k, v, r, scale, d_out, p_drop, seed, out=None):
+    """Gradient of sum(out * d_out) for attn_fwd_dropout (the mask does not depend on the inputs).
+    With W_e = keep_e / (1 - p): dP_e = W_e d_out_u . v_v, dS_e = P_e (dP_e - sum_e' P_e' dP_e'),
+    dv_v += W_e P_e d_out_u; dq, dk, dr from dS as without dropout.  The row term equals
+    d_out_u . out_u; `out` as in attn_bwd."""
+    q, k, v, r, d_out = (np.asarray(a, dtype=np.float64) for a in (q, k, v, r, d_out))
+    B, N, H, d = q.shape
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    dr = np.zeros_like(r)
+    for u in range(N):
+        a, b_ = g.row_ptr[u], g.row_ptr[u + 1]
+        if a == b_:
+            continue
+        src, rl = g.col[a:b_], g.rel[a:b_]
+        kk = k[:, src] + r[rl][None, :, None, :]
+        s = scale * np.einsum("bhc,behc->bhe", q[:, u], kk)
+        s -= s.max(axis=2, keepdims=True)
+        pr = np.exp(s)
+        pr /= pr.sum(axis=2, keepdims=True)
+        w = np.zeros_like(pr)
+        for b in range(B):
+            for h in range(H):
+                w[b, h] = dropout_keep(seed, p_drop, b, h, H, np.full(src.shape, u), src) / (1.0 - p_drop)
+        dp = w * np.einsum("bhc,behc->bhe", d_out[:, u], v[:, src])
+        if out is None:
+            row_term = (pr * dp).sum(axis=2, keepdims=True)
+        else:
+            row_term = (d_out[:, u] * np.asarray(out, dtype=np.float64)[:, u]).sum(axis=2)[:, :, None]
+        ds = pr * (dp - row_term)
+        dq[:, u] = scale * np.einsum("bhe,behc->bhc", ds, kk)
+        dk[:, src] += scale * np.einsum("bhe,bhc->behc", ds, q[:, u])
+        dv[:, src] += np.einsum("bhe,bhc->behc", w * pr, d_out[:, u])
+        np.add.at(dr, rl, scale * np.einsum("bhe,bhc->ec", ds, q[:, u]))
+    return dq, dk, dv, dr

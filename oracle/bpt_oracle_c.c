@@ -126,13 +126,34 @@ void orc_transpose(int64_t n_nodes, const int32_t* row_ptr, const int32_t* col,
 }
 
 /*
+ * Attention dropout mask (see oracle/bpt_oracle.py for the definition): Philox4x32 with 10 rounds,
+ * key = (seed low word, seed high word), counter = (destination, source, batch * H + head, tag);
+ * the edge is kept iff the first output word is >= floor(p * 2^32).  Returns keep / (1 - p).
+ */
+static double dropout_weight(uint64_t seed, double p, int64_t bh, int64_t dst, int64_t src) {
+    if (p <= 0.0) return 1.0;
+    uint32_t c0 = (uint32_t)dst, c1 = (uint32_t)src, c2 = (uint32_t)bh, c3 = 0x42505431u;
+    uint32_t k0 = (uint32_t)(seed & 0xffffffffu), k1 = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    double thr = floor(p * 4294967296.0);
+    if (thr > 4294967295.0) thr = 4294967295.0;
+    return (double)c0 >= thr ? 1.0 / (1.0 - p) : 0.0;
+}
+
+/*
  * Forward.  q,k,v,out: [B, N, H, d] doubles; r: [n_rel, d]; lse: [B, N, H].
  * Only batch entries [b0, b1) are computed (they are independent).
  */
 void orc_attn_fwd(int64_t N, const int32_t* row_ptr, const int32_t* col, const int32_t* rel,
                   int64_t B, int64_t H, int64_t d, int64_t b0, int64_t b1,
                   const double* q, const double* k, const double* v, const double* r, double scale,
-                  double* out, double* lse) {
+                  double* out, double* lse, double p_drop, uint64_t seed) {
     (void)B;
     const int64_t rs = H * d; /* row stride */
 #pragma omp parallel for collapse(2) schedule(dynamic, 1)
@@ -165,7 +186,7 @@ void orc_attn_fwd(int64_t N, const int32_t* row_ptr, const int32_t* col, const i
                 for (int64_t c = 0; c < d; ++c) ou[c] = 0.0;
                 for (int64_t e = a; e < z; ++e) {
                     const double* vv = v + (b * N + col[e]) * rs + h * d;
-                    const double p = s[e - a] / sum;
+                    const double p = s[e - a] / sum * dropout_weight(seed, p_drop, b * H + h, u, col[e]);
                     for (int64_t c = 0; c < d; ++c) ou[c] += p * vv[c];
                 }
                 lse[(b * N + u) * H + h] = mx + log(sum);
@@ -184,7 +205,8 @@ void orc_attn_fwd(int64_t N, const int32_t* row_ptr, const int32_t* col, const i
 void orc_attn_bwd(int64_t N, int64_t n_rel, const int32_t* row_ptr, const int32_t* col, const int32_t* rel,
                   int64_t B, int64_t H, int64_t d, int64_t b0, int64_t b1,
                   const double* q, const double* k, const double* v, const double* r, double scale,
-                  const double* d_out, const double* out_opt, double* dq, double* dk, double* dv, double* dr) {
+                  const double* d_out, const double* out_opt, double* dq, double* dk, double* dv, double* dr,
+                  double p_drop, uint64_t seed) {
     (void)B;
     const int64_t rs = H * d;
     const int64_t nbh = (b1 - b0) * H;
@@ -226,8 +248,8 @@ void orc_attn_bwd(int64_t N, int64_t n_rel, const int32_t* row_ptr, const int32_
                     double acc = 0.0;
                     for (int64_t c = 0; c < d; ++c) acc += gu[c] * vv[c];
                     p[e - a] /= sum;
-                    dp[e - a] = acc;
-                    dot += p[e - a] * acc;
+                    dp[e - a] = acc * dropout_weight(seed, p_drop, b * H + h, u, col[e]); /* dP_e = W_e d_out . v */
+                    dot += p[e - a] * dp[e - a];
                 }
                 if (out_opt) {
                     dot = 0.0;
@@ -240,7 +262,7 @@ void orc_attn_bwd(int64_t N, int64_t n_rel, const int32_t* row_ptr, const int32_
                     for (int64_t c = 0; c < d; ++c) {
                         dq[off_u + c] += scale * ds * (k[off_v + c] + re[c]);
                         dk[off_v + c] += scale * ds * qu[c];
-                        dv[off_v + c] += p[e - a] * gu[c];
+                        dv[off_v + c] += p[e - a] * dropout_weight(seed, p_drop, b * H + h, u, col[e]) * gu[c];
                         drp[(int64_t)rel[e] * d + c] += scale * ds * qu[c];
                     }
                 }

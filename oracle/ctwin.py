@@ -42,9 +42,9 @@ def _load():
         lib.orc_transpose.restype = None
         lib.orc_transpose.argtypes = [i64, p, p, p, p, p]
         lib.orc_attn_fwd.restype = None
-        lib.orc_attn_fwd.argtypes = [i64, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, dbl, p, p]
+        lib.orc_attn_fwd.argtypes = [i64, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, dbl, p, p, dbl, ctypes.c_uint64]
         lib.orc_attn_bwd.restype = None
-        lib.orc_attn_bwd.argtypes = [i64, i64, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, dbl, p, p, p, p, p, p]
+        lib.orc_attn_bwd.argtypes = [i64, i64, p, p, p, i64, i64, i64, i64, i64, p, p, p, p, dbl, p, p, p, p, p, p, dbl, ctypes.c_uint64]
         _lib = lib
     return _lib
 
@@ -83,19 +83,20 @@ def _f64(a):
     return np.ascontiguousarray(a, dtype=np.float64)
 
 
-def attn_fwd(g, q, k, v, r, scale, b0=0, b1=None):
-    """fp64 forward on batch entries [b0, b1); other entries of the outputs stay 0."""
+def attn_fwd(g, q, k, v, r, scale, b0=0, b1=None, p_drop=0.0, seed=0):
+    """fp64 forward on batch entries [b0, b1); other entries of the outputs stay 0.
+    p_drop, seed: attention dropout as defined in oracle/bpt_oracle.py (0 = none)."""
     q, k, v, r = _f64(q), _f64(k), _f64(v), _f64(r)
     B, N, H, d = q.shape
     b1 = B if b1 is None else b1
     out = np.zeros_like(q)
     lse = np.zeros((B, N, H))
     _load().orc_attn_fwd(N, _ptr(g.row_ptr), _ptr(g.col), _ptr(g.rel), B, H, d, b0, b1,
-                         _ptr(q), _ptr(k), _ptr(v), _ptr(r), float(scale), _ptr(out), _ptr(lse))
+                         _ptr(q), _ptr(k), _ptr(v), _ptr(r), float(scale), _ptr(out), _ptr(lse), float(p_drop), int(seed))
     return out, lse
 
 
-def attn_bwd(g, q, k, v, r, scale, d_out, b0=0, b1=None, out=None):
+def attn_bwd(g, q, k, v, r, scale, d_out, b0=0, b1=None, out=None, p_drop=0.0, seed=0):
     """fp64 backward on batch entries [b0, b1); dr sums over those entries only.
     ``out``: optional stored forward output to use in the row term (see the C source)."""
     q, k, v, r, d_out = _f64(q), _f64(k), _f64(v), _f64(r), _f64(d_out)
@@ -107,7 +108,7 @@ def attn_bwd(g, q, k, v, r, scale, d_out, b0=0, b1=None, out=None):
     _load().orc_attn_bwd(N, r.shape[0], _ptr(g.row_ptr), _ptr(g.col), _ptr(g.rel), B, H, d, b0, b1,
                          _ptr(q), _ptr(k), _ptr(v), _ptr(r), float(scale), _ptr(d_out),
                          None if out is None else _ptr(_out),
-                         _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dr))
+                         _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dr), float(p_drop), int(seed))
     return dq, dk, dv, dr
 
 
