@@ -166,6 +166,34 @@ bpt_status bpt_attn_bwd_varlen(const bpt_graph* g, int32_t B, int32_t H, int32_t
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The general form of the two operations: optional sequence lengths (as for the _varlen entry points,
+ * NULL = all n) and attention dropout (App. A.1 of the paper lists an attention dropout rate for
+ * every experiment; the way the masks are drawn is the library's).  With 0 < dropout_p < 1 every edge
+ * weight of every (batch entry, head) is kept with probability 1 - dropout_p and divided by
+ * 1 - dropout_p, after the softmax and before the product with v; lse is that of the softmax.
+ * The mask is a pure function of (dropout_seed, batch entry, head, destination node, source node):
+ * Philox4x32 with 10 rounds, key = (low, high) word of the seed, counter = (destination, source,
+ * batch entry * H + head, 0x42505431), edge kept iff the first output word >= floor(dropout_p * 2^32).
+ * The backward rebuilds it from the same options (nothing is stored); pass the options the forward had.
+ * `opt` is a host pointer; NULL means no lengths and no dropout.  dropout_p outside [0, 1): INVALID_ARG.
+ */
+typedef struct {
+    const int32_t* lengths; /* device [B] or NULL */
+    float dropout_p;
+    uint64_t dropout_seed;
+} bpt_attn_options;
+
+bpt_status bpt_attn_fwd_ex(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                           const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                           const bpt_attn_options* opt, void* out, float* lse,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+bpt_status bpt_attn_bwd_ex(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                           const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                           const bpt_attn_options* opt, const void* out, const float* lse, const void* d_out,
+                           void* dq, void* dk, void* dv, float* d_rel,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Backward pass for callers that must not allocate device memory (the paper has no
  * counterpart; this is a deployment convenience).
  *

@@ -19,7 +19,8 @@ BPT_F32, BPT_BF16 = 0, 1
 
 EXPORTS = ("bpt_graph_dims_query", "bpt_build_graph", "bpt_attn_workspace_bytes", "bpt_attn_fwd",
            "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end",
-           "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch", "bpt_attn_fwd_varlen", "bpt_attn_bwd_varlen")
+           "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch", "bpt_attn_fwd_varlen", "bpt_attn_bwd_varlen",
+           "bpt_attn_fwd_ex", "bpt_attn_bwd_ex")
 
 
 class BptError(RuntimeError):
@@ -38,6 +39,10 @@ class GraphStruct(ctypes.Structure):
     _fields_ = [("row_ptr", ctypes.c_void_p), ("col", ctypes.c_void_p), ("rel", ctypes.c_void_p),
                 ("t_ptr", ctypes.c_void_p), ("t_dst", ctypes.c_void_p), ("t_eid", ctypes.c_void_p),
                 ("dims", GraphDims)]
+
+
+class AttnOptions(ctypes.Structure):
+    _fields_ = [("lengths", ctypes.c_void_p), ("dropout_p", ctypes.c_float), ("dropout_seed", ctypes.c_uint64)]
 
 
 _lib = None
@@ -70,6 +75,12 @@ def load_library() -> ctypes.CDLL:
         lib.bpt_attn_bwd_varlen.restype = ctypes.c_int
         lib.bpt_attn_bwd_varlen.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
                                             vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.bpt_attn_fwd_ex.restype = ctypes.c_int
+        lib.bpt_attn_fwd_ex.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
+                                        ctypes.POINTER(AttnOptions), vp, vp, vp, sz, vp]
+        lib.bpt_attn_bwd_ex.restype = ctypes.c_int
+        lib.bpt_attn_bwd_ex.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
+                                        ctypes.POINTER(AttnOptions), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.bpt_static_scratch_bytes.restype = sz
         lib.bpt_static_scratch_bytes.argtypes = []
         lib.bpt_attn_bwd_static_scratch.restype = ctypes.c_int
@@ -175,9 +186,11 @@ def _check_lengths(lengths, q):
         raise ValueError("lengths must be a contiguous int32 tensor [B] on the device of q")
 
 
-def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, workspace=None, lengths=None):
+def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, workspace=None, lengths=None,
+                 dropout_p: float = 0.0, dropout_seed: int = 0):
     """Returns (out [B,N,H,d], lse [B,N,H] fp32).  With `lengths` (int32 [B] on the device) batch entry b
-    has lengths[b] real tokens; see bpt_attn_fwd_varlen in include/bpt.h."""
+    has lengths[b] real tokens; with dropout_p > 0 the attention weights are dropped (mask defined by
+    dropout_seed); see bpt_attn_fwd_varlen / bpt_attn_fwd_ex in include/bpt.h."""
     lib = load_library()
     _check_layout(g, q, k, v)
     B, N, H, d = q.shape
@@ -191,7 +204,14 @@ def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, w
         if workspace is None and need:
             workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
         ws_n = 0 if workspace is None else workspace.numel()
-        if lengths is None:
+        if dropout_p:
+            if lengths is not None:
+                _check_lengths(lengths, q)
+            opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed))
+            _check(lib.bpt_attn_fwd_ex(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
+                                       float(scale), ctypes.byref(opt), _ptr(out), _ptr(lse), _ptr(workspace), ws_n,
+                                       _stream()), "bpt_attn_fwd_ex")
+        elif lengths is None:
             _check(lib.bpt_attn_fwd(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
                                     float(scale), _ptr(out), _ptr(lse), _ptr(workspace), ws_n, _stream()), "bpt_attn_fwd")
         else:
@@ -203,8 +223,9 @@ def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, w
 
 
 def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, workspace=None,
-                 dq=None, dk=None, dv=None, d_rel=None, lengths=None):
-    """Returns (dq, dk, dv [B,N,H,d], d_rel [n_rel, d] fp32).  `lengths` as for bpt_attn_fwd."""
+                 dq=None, dk=None, dv=None, d_rel=None, lengths=None, dropout_p: float = 0.0, dropout_seed: int = 0):
+    """Returns (dq, dk, dv [B,N,H,d], d_rel [n_rel, d] fp32).  `lengths`, `dropout_p`, `dropout_seed` as for
+    bpt_attn_fwd (pass what the forward had)."""
     lib = load_library()
     _check_layout(g, q, k, v, out, d_out)
     B, N, H, d = q.shape
@@ -218,7 +239,14 @@ def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, work
         if workspace is None and need:
             workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
         ws_n = 0 if workspace is None else workspace.numel()
-        if lengths is None:
+        if dropout_p:
+            if lengths is not None:
+                _check_lengths(lengths, q)
+            opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed))
+            _check(lib.bpt_attn_bwd_ex(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
+                                       float(scale), ctypes.byref(opt), _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq),
+                                       _ptr(dk), _ptr(dv), _ptr(d_rel), _ptr(workspace), ws_n, _stream()), "bpt_attn_bwd_ex")
+        elif lengths is None:
             _check(lib.bpt_attn_bwd(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
                                     float(scale), _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq), _ptr(dk), _ptr(dv),
                                     _ptr(d_rel), _ptr(workspace), ws_n, _stream()), "bpt_attn_bwd")

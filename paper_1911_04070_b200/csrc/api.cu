@@ -23,8 +23,8 @@ extern "C" size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_
 
 static bpt_status attn_fwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                 const void* q, const void* k, const void* v, const void* rel_emb, float scale,
-                                const int32_t* lengths, void* out, float* lse, void* workspace, size_t workspace_bytes,
-                                void* cuda_stream) {
+                                const int32_t* lengths, DropoutParams drop, void* out, float* lse, void* workspace,
+                                size_t workspace_bytes, void* cuda_stream) {
     const bpt_status s = check_problem(g, B, H, d, dtype, false);
     if (s != BPT_OK) return s;
     if (!q || !k || !v || !rel_emb || !out || !lse) return BPT_ERR_INVALID_ARG;
@@ -34,7 +34,7 @@ static bpt_status attn_fwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_
     p.g = g;
     tree_params_from_dims(g->dims, &p.tree);
     p.B = B; p.H = H; p.d = d; p.dtype = dtype;
-    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths; p.drop = drop;
     p.out = out; p.lse = lse;
     p.workspace = workspace; p.workspace_bytes = workspace_bytes;
     p.stream = (cudaStream_t)cuda_stream;
@@ -44,7 +44,7 @@ static bpt_status attn_fwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_
 extern "C" bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                    const void* q, const void* k, const void* v, const void* rel_emb, float scale,
                                    void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
-    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, out, lse, workspace, workspace_bytes, cuda_stream);
+    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, make_dropout(0.f, 0), out, lse, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" bpt_status bpt_attn_fwd_varlen(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
@@ -52,12 +52,24 @@ extern "C" bpt_status bpt_attn_fwd_varlen(const bpt_graph* g, int32_t B, int32_t
                                           const int32_t* lengths, void* out, float* lse, void* workspace,
                                           size_t workspace_bytes, void* cuda_stream) {
     if (!lengths) return BPT_ERR_INVALID_ARG;
-    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, out, lse, workspace, workspace_bytes, cuda_stream);
+    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, make_dropout(0.f, 0), out, lse, workspace, workspace_bytes, cuda_stream);
+}
+
+static bool options_ok(const bpt_attn_options* opt) { return !opt || (opt->dropout_p >= 0.f && opt->dropout_p < 1.f); }
+
+extern "C" bpt_status bpt_attn_fwd_ex(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                      const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                      const bpt_attn_options* opt, void* out, float* lse, void* workspace,
+                                      size_t workspace_bytes, void* cuda_stream) {
+    if (!options_ok(opt)) return BPT_ERR_INVALID_ARG;
+    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, opt ? opt->lengths : nullptr,
+                         opt ? make_dropout(opt->dropout_p, opt->dropout_seed) : make_dropout(0.f, 0), out, lse, workspace,
+                         workspace_bytes, cuda_stream);
 }
 
 static bpt_status attn_bwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                 const void* q, const void* k, const void* v, const void* rel_emb, float scale,
-                                const int32_t* lengths, const void* out, const float* lse, const void* d_out,
+                                const int32_t* lengths, DropoutParams drop, const void* out, const float* lse, const void* d_out,
                                 void* dq, void* dk, void* dv, float* d_rel,
                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
     const bpt_status s = check_problem(g, B, H, d, dtype, true);
@@ -69,7 +81,7 @@ static bpt_status attn_bwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_
     p.g = g;
     tree_params_from_dims(g->dims, &p.tree);
     p.B = B; p.H = H; p.d = d; p.dtype = dtype;
-    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths; p.drop = drop;
     p.out = const_cast<void*>(out); p.lse = const_cast<float*>(lse);
     p.d_out = d_out; p.dq = dq; p.dk = dk; p.dv = dv; p.d_rel = d_rel;
     p.workspace = workspace; p.workspace_bytes = workspace_bytes;
@@ -82,7 +94,7 @@ extern "C" bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int
                                    const void* out, const float* lse, const void* d_out,
                                    void* dq, void* dk, void* dv, float* d_rel,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
-    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, out, lse, d_out, dq, dk, dv, d_rel,
+    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, make_dropout(0.f, 0), out, lse, d_out, dq, dk, dv, d_rel,
                          workspace, workspace_bytes, cuda_stream);
 }
 
@@ -92,8 +104,19 @@ extern "C" bpt_status bpt_attn_bwd_varlen(const bpt_graph* g, int32_t B, int32_t
                                           void* dq, void* dk, void* dv, float* d_rel,
                                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!lengths) return BPT_ERR_INVALID_ARG;
-    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, out, lse, d_out, dq, dk, dv, d_rel,
+    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, make_dropout(0.f, 0), out, lse, d_out, dq, dk, dv, d_rel,
                          workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" bpt_status bpt_attn_bwd_ex(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                      const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                      const bpt_attn_options* opt, const void* out, const float* lse, const void* d_out,
+                                      void* dq, void* dk, void* dv, float* d_rel,
+                                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!options_ok(opt)) return BPT_ERR_INVALID_ARG;
+    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, opt ? opt->lengths : nullptr,
+                         opt ? make_dropout(opt->dropout_p, opt->dropout_seed) : make_dropout(0.f, 0), out, lse, d_out,
+                         dq, dk, dv, d_rel, workspace, workspace_bytes, cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------

@@ -53,7 +53,7 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
                const T* __restrict__ out, const float* __restrict__ lse, const T* __restrict__ d_out,
                T* __restrict__ dq, float* __restrict__ ws_p, float* __restrict__ ws_ds,
                int N, int row0, int nrows, int H, int ngroups, int64_t e_first, int64_t E, float scale,
-               const int32_t* __restrict__ lengths) {
+               const int32_t* __restrict__ lengths, DropoutParams drop) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
@@ -119,8 +119,11 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
                 }
                 s = M::head_sum(s);
                 dp = M::head_sum(dp);
-                const float p = fast_exp2(fmaf(s, sc2, -lse2));
-                const float ds = p * (dp - delta);
+                float p = fast_exp2(fmaf(s, sc2, -lse2));
+                // dropout: dP = W d_out.v and the weight that reaches dv is W P; dS keeps the undropped P
+                const float wgt = drop.thr ? dropout_weight(drop, (uint32_t)(b * H + hc), (uint32_t)u, (uint32_t)c) : 1.f;
+                const float ds = p * (dp * wgt - delta);
+                p *= wgt;
 #pragma unroll
                 for (int x = 0; x < EPL; ++x) acc[x] = fmaf(ds, kk[x], acc[x]);
                 if (sub == 0 && head_ok) {
@@ -376,7 +379,7 @@ static bpt_status launch_bwd_rows(const AttnProblem& p) {
     const size_t smem_a = nw > 1 ? (size_t)nw * 32 * M::EPL * sizeof(float) : 0;
     bwd_dst_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem_a, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, 0, N, p.H, ngroups, 0, E, p.scale, p.lengths);
+        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, 0, N, p.H, ngroups, 0, E, p.scale, p.lengths, p.drop);
     trace_mark(p.stream, "bwd_dst");
 
     const size_t smem_b = nw > 1 ? (size_t)nw * 32 * (2 * M::EPL) * sizeof(float) : 0;

@@ -94,7 +94,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 const __nv_bfloat16* __restrict__ out, const float* __restrict__ lse,
                 const __nv_bfloat16* __restrict__ d_out, __nv_bfloat16* __restrict__ dq,
                 int2* __restrict__ tile_range, float* __restrict__ slabs, float* __restrict__ drel_part,
-                int H, int pair0, float scale, const int32_t* __restrict__ lengths) {
+                int H, int pair0, float scale, const int32_t* __restrict__ lengths, DropoutParams drop) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* q_s = smem;
     unsigned char* g_s = q_s + BwdTileSmem::q_bytes;   // d_out tile
@@ -301,7 +301,10 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                         const int off = side ? m - lo_r[hh] : hi_r[hh] - m;
                         const float bias = qr_w[(g + hh * 8) * kQrStride + off];
                         p = fast_exp2(fmaf(s[j][e] + bias, scale_log2e, -lse_r[hh]));
-                        d = p * (dp[j][e] - del_r[hh]);
+                        // dropout: dP = W d_out.v and the weight that reaches dv is W P; dS keeps the undropped P
+                        const float wgt = drop.thr ? dropout_weight(drop, (uint32_t)pair, (uint32_t)(t0 + r0 + g + hh * 8), (uint32_t)(gm.id_base + m)) : 1.f;
+                        d = p * (dp[j][e] * wgt - del_r[hh]);
+                        p *= wgt;
                         *reinterpret_cast<__nv_bfloat16*>(sk_s + (r0 + g + hh * 8) * kSkewStride + off * 2) = __float2bfloat16_rn(d);
                     }
                     pv[e] = p; dv[e] = d;
@@ -618,7 +621,7 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
         bwd_tile_kernel<<<dim3(tiles, np), kBwdThreads, smem, p.stream>>>(
             t, plan, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
             (const __nv_bfloat16*)p.rel_emb, (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out,
-            (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale, p.lengths);
+            (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale, p.lengths, p.drop);
         trace_mark(p.stream, "bwd_tile");
         const int64_t warps = (int64_t)np * N;
         bwd_gather_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, p.stream>>>(

@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(256)
 fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col, const int32_t* __restrict__ rel,
                 const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
                 T* __restrict__ out, float* __restrict__ lse, int N, int row0, int nrows, int H, int ngroups,
-                float scale_log2e, const int32_t* __restrict__ lengths) {
+                float scale_log2e, const int32_t* __restrict__ lengths, DropoutParams drop) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
@@ -52,10 +52,11 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
         const int cnt = min(U, z - e0);
         int my_c = 0, my_r = 0;
         if (lane < cnt) { my_c = col[e0 + lane]; my_r = rel[e0 + lane]; }
-        float s[U], vv[U][EPL];
+        float s[U], vv[U][EPL], wgt[U];
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             const int c = __shfl_sync(0xffffffffu, my_c, j), rr = __shfl_sync(0xffffffffu, my_r, j);
+            wgt[j] = (drop.thr && j < cnt) ? dropout_weight(drop, (uint32_t)(b * H + hc), (uint32_t)u, (uint32_t)c) : 1.f;
             if (j < cnt && (len >= n_tok || node_first_token(n_tok, c) < len)) {
                 float kk[EPL], rv[EPL];
                 M::load(k + boff + (size_t)c * rs, sub, kk);
@@ -86,8 +87,9 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
         for (int j = 0; j < U; ++j) {
             const float p = fast_exp2(s[j] - m_ref);
             l += p;
+            const float pw = p * wgt[j];  // dropout acts on the weight that reaches V, not on the softmax sum
 #pragma unroll
-            for (int x = 0; x < EPL; ++x) acc[x] = fmaf(p, vv[j][x], acc[x]);
+            for (int x = 0; x < EPL; ++x) acc[x] = fmaf(pw, vv[j][x], acc[x]);
         }
         m = m_new;
     }
@@ -143,7 +145,7 @@ static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows) {
     const size_t smem = nw > 1 ? (size_t)nw * 32 * (2 + M::EPL) * sizeof(float) : 0;
     fwd_rows_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e, p.lengths);
+        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e, p.lengths, p.drop);
     trace_mark(p.stream, "fwd_rows");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }

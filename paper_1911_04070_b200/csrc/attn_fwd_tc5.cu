@@ -79,12 +79,14 @@ __device__ __forceinline__ void quad_barrier(int quad) {
     }
 }
 
+template <bool kDrop>  // attention dropout compiled in or out
 __global__ void __launch_bounds__(kTcThreads, 1)
 fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
                const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
                __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int* __restrict__ status,
-               int H, float scale_log2e, const int32_t* __restrict__ lengths, const __grid_constant__ CUtensorMap tm_k,
+               int H, float scale_log2e, const int32_t* __restrict__ lengths, DropoutParams drop,
+               const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_r) {
     extern __shared__ unsigned char smem_raw[];
     // the swizzle pattern is a function of the address bits, so the tiles must start 1024-aligned
@@ -369,9 +371,14 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
                     uint32_t pk[4];
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {
-                        const float p0 = ex2(__uint_as_float(sv[p][2 * x]) - m_ref);
-                        const float p1 = ex2(__uint_as_float(sv[p][2 * x + 1]) - m_ref);
+                        float p0 = ex2(__uint_as_float(sv[p][2 * x]) - m_ref);
+                        float p1 = ex2(__uint_as_float(sv[p][2 * x + 1]) - m_ref);
                         l4[x] += p0 + p1;
+                        if constexpr (kDrop) {  // the weights that reach V are dropped, the softmax sum is not
+                            const uint32_t src = (uint32_t)(node_id(t.n, level, 0) + base + c0 + p * 32 + part * kCols + 2 * x);
+                            p0 *= dropout_weight(drop, (uint32_t)(b * H + h), (uint32_t)(t0 + row), src);
+                            p1 *= dropout_weight(drop, (uint32_t)(b * H + h), (uint32_t)(t0 + row), src + 1);
+                        }
                         pk[x] = pack_bf16(p0, p1);
                     }
                     const int ci = ch0 + p * 4 + part;  // 16-byte chunk (8 keys) of the P row
@@ -480,7 +487,8 @@ bpt_status launch_fwd_tc5(const AttnProblem& p, int* status) {
     context_levels(p.tree, &n_left, &n_right);
     const size_t smem = FwdTcSmem::bytes(n_left + n_right);
     if (smem > 227 * 1024 || p.H > 65535 || p.B > 65535) return BPT_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(fwd_tc5_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    auto kernel = p.drop.thr ? fwd_tc5_kernel<true> : fwd_tc5_kernel<false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return BPT_ERR_CUDA;
     alignas(64) CUtensorMap tm_k, tm_v, tm_r;
     const int N = 2 * p.tree.n - 1;
@@ -488,10 +496,10 @@ bpt_status launch_fwd_tc5(const AttnProblem& p, int* status) {
         !rel_rows_map(&tm_r, p.rel_emb, p.g->dims.n_rel))
         return BPT_ERR_CUDA;
     const dim3 grid(p.tree.n / kTcTokens, p.H, p.B);
-    fwd_tc5_kernel<<<grid, kTcThreads, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q,
-                                                         (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
-                                                         (const __nv_bfloat16*)p.rel_emb, (__nv_bfloat16*)p.out, p.lse,
-                                                         status, p.H, p.scale * kLog2e, p.lengths, tm_k, tm_v, tm_r);
+    kernel<<<grid, kTcThreads, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q,
+                                                 (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
+                                                 (const __nv_bfloat16*)p.rel_emb, (__nv_bfloat16*)p.out, p.lse,
+                                                 status, p.H, p.scale * kLog2e, p.lengths, p.drop, tm_k, tm_v, tm_r);
     trace_mark(p.stream, "fwd_tc5");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }

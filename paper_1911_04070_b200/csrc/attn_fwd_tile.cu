@@ -39,12 +39,13 @@ struct FwdTileSmem {
     static size_t bytes(int chunks) { return (size_t)fixed + (size_t)chunks * (kTileTokens * 8 + 8); }
 };
 
+template <bool kDrop>  // attention dropout compiled in or out: the plain kernel carries none of it
 __global__ void __launch_bounds__(128)
 fwd_tile_kernel(TreeParams t, int n_left, int n_right,
                 const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                 const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
                 __nv_bfloat16* __restrict__ out, float* __restrict__ lse, int H, float scale_log2e,
-                const int32_t* __restrict__ lengths) {
+                const int32_t* __restrict__ lengths, DropoutParams drop) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* q_s = smem;
     unsigned char* k_s = q_s + FwdTileSmem::q_bytes;
@@ -110,6 +111,15 @@ fwd_tile_kernel(TreeParams t, int n_left, int n_right,
                 dot[hh] = fmaf(__uint_as_float(qq & 0xffff0000u), __uint_as_float(kk & 0xffff0000u) + r_hi, dot[hh]);
                 o[nt][hh * 2] = __uint_as_float(vv << 16);
                 o[nt][hh * 2 + 1] = __uint_as_float(vv & 0xffff0000u);
+            }
+        }
+        if constexpr (kDrop) {  // dropout on the self loop's weight (the softmax sum keeps the undropped weight)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const uint32_t tok = (uint32_t)(t0 + r0 + g + hh * 8);
+                const float wgt = dropout_weight(drop, (uint32_t)(b * H + h), tok, tok);
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) { o[nt][hh * 2] *= wgt; o[nt][hh * 2 + 1] *= wgt; }
             }
         }
 #pragma unroll
@@ -233,10 +243,16 @@ fwd_tile_kernel(TreeParams t, int n_left, int n_right,
             uint32_t pa[2][4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const float p0 = ex2(s[j][0] - m_run[0]), p1 = ex2(s[j][1] - m_run[0]);
-                const float p2 = ex2(s[j][2] - m_run[1]), p3 = ex2(s[j][3] - m_run[1]);
+                float p0 = ex2(s[j][0] - m_run[0]), p1 = ex2(s[j][1] - m_run[0]);
+                float p2 = ex2(s[j][2] - m_run[1]), p3 = ex2(s[j][3] - m_run[1]);
                 l_run[0] += p0 + p1;
                 l_run[1] += p2 + p3;
+                if constexpr (kDrop) {  // the weights that reach V are dropped, the softmax sum is not
+                    const uint32_t bh = (uint32_t)(b * H + h), src = (uint32_t)(id_base + base + kb + j * 8 + c2);
+                    const uint32_t d0 = (uint32_t)(t0 + r0 + g), d1 = d0 + 8;
+                    p0 *= dropout_weight(drop, bh, d0, src); p1 *= dropout_weight(drop, bh, d0, src + 1);
+                    p2 *= dropout_weight(drop, bh, d1, src); p3 *= dropout_weight(drop, bh, d1, src + 1);
+                }
                 pa[j >> 1][(j & 1) * 2] = pack_bf16(p0, p1);
                 pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
             }
@@ -287,14 +303,15 @@ bpt_status launch_fwd_tile(const AttnProblem& p) {
     int n_left, n_right;
     context_levels(p.tree, &n_left, &n_right);
     const size_t smem = FwdTileSmem::bytes(n_left + n_right);
-    if (cudaFuncSetAttribute(fwd_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+    auto kernel = p.drop.thr ? fwd_tile_kernel<true> : fwd_tile_kernel<false>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
         return BPT_ERR_CUDA;
     if (smem > 200 * 1024 || p.H > 65535 || p.B > 65535) return BPT_ERR_UNSUPPORTED;
     const dim3 grid(p.tree.n / kTileTokens, p.H, p.B);
-    fwd_tile_kernel<<<grid, 128, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q,
-                                                   (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
-                                                   (const __nv_bfloat16*)p.rel_emb, (__nv_bfloat16*)p.out, p.lse, p.H,
-                                                   p.scale * kLog2e, p.lengths);
+    kernel<<<grid, 128, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q,
+                                          (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
+                                          (const __nv_bfloat16*)p.rel_emb, (__nv_bfloat16*)p.out, p.lse, p.H,
+                                          p.scale * kLog2e, p.lengths, p.drop);
     trace_mark(p.stream, "fwd_tile");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }

@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kSpanThreads)
 fwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                 const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
                 __nv_bfloat16* __restrict__ out, float* __restrict__ lse, float* __restrict__ ext_part,
-                int H, int n_ext, float scale_log2e, const int32_t* __restrict__ lengths) {
+                int H, int n_ext, float scale_log2e, const int32_t* __restrict__ lengths, DropoutParams drop) {
     __shared__ __align__(128) unsigned char qs_s[kSpanRows * 128];
     __shared__ __align__(128) unsigned char k_s[kTileTokens * 128];
     __shared__ __align__(128) unsigned char v_s[kTileTokens * 128];
@@ -173,10 +173,16 @@ fwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
     uint32_t pa[4][4];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const float p0 = fast_exp2(s[j][0] - m_use[0]), p1 = fast_exp2(s[j][1] - m_use[0]);
-        const float p2 = fast_exp2(s[j][2] - m_use[1]), p3 = fast_exp2(s[j][3] - m_use[1]);
+        float p0 = fast_exp2(s[j][0] - m_use[0]), p1 = fast_exp2(s[j][1] - m_use[0]);
+        float p2 = fast_exp2(s[j][2] - m_use[1]), p3 = fast_exp2(s[j][3] - m_use[1]);
         l_run[0] += p0 + p1;
         l_run[1] += p2 + p3;
+        if (drop.thr) {  // the weights that reach V are dropped, the softmax sum is not
+            const uint32_t bh = (uint32_t)(b * H + h), src = (uint32_t)(t0 + j * 8 + c2);
+            const uint32_t d0 = (uint32_t)meta.node[r0 + g], d1 = (uint32_t)meta.node[r0 + g + 8];
+            p0 *= dropout_weight(drop, bh, d0, src); p1 *= dropout_weight(drop, bh, d0, src + 1);
+            p2 *= dropout_weight(drop, bh, d1, src); p3 *= dropout_weight(drop, bh, d1, src + 1);
+        }
         pa[j >> 1][(j & 1) * 2] = pack_bf16(p0, p1);
         pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
     }
@@ -255,11 +261,12 @@ fwd_span_merge_kernel(TreeParams t, const float* __restrict__ ext_part, __nv_bfl
     for (int x = lane; x < nT; x += 32) mx = fmaxf(mx, base[(size_t)x * stride]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (mx == -INFINITY) mx = 0.f;  // a span without real tokens: every partial is empty (2^-inf = 0 below)
     float l = 0.f, a0 = 0.f, a1 = 0.f;
 #pragma unroll 4
     for (int x = 0; x < nT; ++x) {
         const float* p = base + (size_t)x * stride;
-        const float f = mx == -INFINITY ? 0.f : fast_exp2(p[0] - mx);
+        const float f = fast_exp2(p[0] - mx);
         const float2 a = *reinterpret_cast<const float2*>(p + 2 + lane * 2);
         l = fmaf(p[1], f, l);
         a0 = fmaf(a.x, f, a0);
@@ -280,7 +287,7 @@ bwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
                 const __nv_bfloat16* __restrict__ out, const float* __restrict__ lse,
                 const __nv_bfloat16* __restrict__ d_out, __nv_bfloat16* __restrict__ dq,
                 float* __restrict__ ext_dq, float* __restrict__ aff_slab,
-                int H, int pair0, int n_ext, float scale, const int32_t* __restrict__ lengths) {
+                int H, int pair0, int n_ext, float scale, const int32_t* __restrict__ lengths, DropoutParams drop) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* qs_s = smem;
     unsigned char* gs_s = qs_s + kSpanRows * 128;
@@ -399,7 +406,10 @@ bwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
                 float p = 0.f, d = 0.f;
                 if (ok) {
                     p = fast_exp2(fmaf(s[j][e], scale_log2e, bias_r[hh] - lse_r[hh]));
-                    d = p * (dp[j][e] - del_r[hh]);
+                    // dropout: dP = W d_out.v and the weight that reaches dv is W P; dS keeps the undropped P
+                    const float wgt = drop.thr ? dropout_weight(drop, (uint32_t)(b * H + h), (uint32_t)meta.node[r0 + g + hh * 8], (uint32_t)(t0 + m)) : 1.f;
+                    d = p * (dp[j][e] * wgt - del_r[hh]);
+                    p *= wgt;
                 }
                 pv[e] = p; dv[e] = d;
                 rowsum[hh] += d;
@@ -551,7 +561,7 @@ bpt_status launch_fwd_span(const AttnProblem& p) {
     float* ext = (float*)p.workspace;
     fwd_span_kernel<<<dim3(tiles, p.H, p.B), kSpanThreads, 0, p.stream>>>(
         t, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v, (const __nv_bfloat16*)p.rel_emb,
-        (__nv_bfloat16*)p.out, p.lse, ext, p.H, n_ext, p.scale * kLog2e, p.lengths);
+        (__nv_bfloat16*)p.out, p.lse, ext, p.H, n_ext, p.scale * kLog2e, p.lengths, p.drop);
     trace_mark(p.stream, "fwd_span");
     if (n_ext > 0) {
         const int64_t warps = (int64_t)p.B * p.H * (tiles - 1);
@@ -576,7 +586,7 @@ bpt_status launch_bwd_span(const AttnProblem& p, int pair0, int n_pairs, float* 
     bwd_span_kernel<<<dim3(tiles, n_pairs), kSpanThreads, kBwdSpanSmem, p.stream>>>(
         t, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v, (const __nv_bfloat16*)p.rel_emb,
         (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out, (__nv_bfloat16*)p.dq, ext_dq, aff_slab,
-        p.H, pair0, n_ext, p.scale, p.lengths);
+        p.H, pair0, n_ext, p.scale, p.lengths, p.drop);
     trace_mark(p.stream, "bwd_span");
     if (n_ext > 0) {
         const int64_t warps = (int64_t)n_pairs * (tiles - 1);

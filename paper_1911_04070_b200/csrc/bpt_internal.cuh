@@ -7,6 +7,7 @@
 
 #include "../../include/bpt.h"
 #include "bpt_tree.cuh"
+#include "dropout.cuh"
 
 namespace bpt {
 
@@ -20,6 +21,7 @@ struct AttnProblem {
     bpt_dtype dtype;
     const void *q, *k, *v, *rel_emb;
     const int32_t* lengths;  // [B] real tokens per batch entry, or nullptr: all n (see bpt_attn_fwd_varlen)
+    DropoutParams drop;      // attention dropout (thr = 0: none)
     float scale;
     // forward outputs / backward inputs
     void* out;

@@ -19,28 +19,30 @@ class _GraphSelfAttention(torch.autograd.Function):
     """out = GSA(q, k, v, rel_emb) over the BPT graph; backward through bpt_attn_bwd."""
 
     @staticmethod
-    def forward(ctx, q, k, v, rel_emb, g, scale, lengths):
+    def forward(ctx, q, k, v, rel_emb, g, scale, lengths, dropout_p, dropout_seed):
         q, k, v, rel_emb = q.contiguous(), k.contiguous(), v.contiguous(), rel_emb.contiguous()
-        out, lse = binding.bpt_attn_fwd(g, q, k, v, rel_emb, scale, lengths=lengths)
+        out, lse = binding.bpt_attn_fwd(g, q, k, v, rel_emb, scale, lengths=lengths, dropout_p=dropout_p,
+                                        dropout_seed=dropout_seed)
         ctx.save_for_backward(q, k, v, rel_emb, out, lse)
-        ctx.g, ctx.scale, ctx.lengths = g, scale, lengths
+        ctx.g, ctx.scale, ctx.lengths, ctx.drop = g, scale, lengths, (dropout_p, dropout_seed)
         return out
 
     @staticmethod
     def backward(ctx, d_out):
         q, k, v, rel_emb, out, lse = ctx.saved_tensors
         dq, dk, dv, d_rel = binding.bpt_attn_bwd(ctx.g, q, k, v, rel_emb, ctx.scale, out, lse, d_out.contiguous(),
-                                                 lengths=ctx.lengths)
-        return dq, dk, dv, d_rel.to(rel_emb.dtype), None, None, None
+                                                 lengths=ctx.lengths, dropout_p=ctx.drop[0], dropout_seed=ctx.drop[1])
+        return dq, dk, dv, d_rel.to(rel_emb.dtype), None, None, None, None, None
 
 
-def graph_self_attention(g: binding.Graph, q, k, v, rel_emb, scale=None, lengths=None):
+def graph_self_attention(g: binding.Graph, q, k, v, rel_emb, scale=None, lengths=None, dropout_p=0.0, dropout_seed=0):
     """Differentiable graph self-attention with tree relative positions (Sec. 3.1, 3.4).
 
     q, k, v: [B, 2n-1, H, d] (float32 or bfloat16, on the graph's device); rel_emb: [n_rel, d], shared
-    by the heads; lengths: optional int32 [B].  Returns [B, 2n-1, H, d]."""
+    by the heads; lengths: optional int32 [B]; dropout_p / dropout_seed: attention dropout (the mask is a
+    function of the seed, so the backward pass rebuilds it).  Returns [B, 2n-1, H, d]."""
     scale = 1.0 / math.sqrt(q.shape[-1]) if scale is None else float(scale)
-    return _GraphSelfAttention.apply(q, k, v, rel_emb, g, scale, lengths)
+    return _GraphSelfAttention.apply(q, k, v, rel_emb, g, scale, lengths, float(dropout_p), int(dropout_seed))
 
 
 class BPTLayer(nn.Module):
@@ -49,8 +51,10 @@ class BPTLayer(nn.Module):
     H holds the states of all 2n-1 nodes.  The relation embeddings are a parameter of the layer
     (Sec. 3.4: not shared between layers, shared between the heads)."""
 
-    def __init__(self, g: binding.Graph, d_model: int, n_heads: int, d_ff: int, rel_std: float = 0.02):
+    def __init__(self, g: binding.Graph, d_model: int, n_heads: int, d_ff: int, rel_std: float = 0.02,
+                 attn_dropout: float = 0.0):
         super().__init__()
+        self.attn_dropout = attn_dropout
         if d_model % n_heads:
             raise ValueError("d_model must be a multiple of n_heads")
         self.g, self.h, self.dh = g, n_heads, d_model // n_heads
@@ -62,8 +66,10 @@ class BPTLayer(nn.Module):
     def forward(self, h, lengths=None):
         B, N, D = h.shape
         split = lambda x: x.view(B, N, self.h, self.dh)
+        p_drop = self.attn_dropout if self.training else 0.0
+        seed = int(torch.randint(0, 2 ** 62, (1,)).item()) if p_drop else 0   # a fresh mask per call, from torch's CPU generator
         a = graph_self_attention(self.g, split(self.wq(h)), split(self.wk(h)), split(self.wv(h)),
-                                 self.rel_emb.to(h.dtype), lengths=lengths)
+                                 self.rel_emb.to(h.dtype), lengths=lengths, dropout_p=p_drop, dropout_seed=seed)
         z = self.norm1(h + self.wo(a.reshape(B, N, D)))
         return self.norm2(z + self.ff2(torch.relu(self.ff1(z))))
 
@@ -76,11 +82,11 @@ class BPTEncoder(nn.Module):
     (language modelling, translation), "root" the root node's state [B, D] (classification)."""
 
     def __init__(self, n: int, k: int, d_model: int, n_heads: int, d_ff: int, n_layers: int, left_only: bool = False,
-                 device="cuda"):
+                 device="cuda", attn_dropout: float = 0.0):
         super().__init__()
         self.n = n
         self.g = binding.bpt_build_graph(n, k, binding.BPT_LEFT_ONLY if left_only else 0, device=device)
-        self.layers = nn.ModuleList(BPTLayer(self.g, d_model, n_heads, d_ff) for _ in range(n_layers))
+        self.layers = nn.ModuleList(BPTLayer(self.g, d_model, n_heads, d_ff, attn_dropout=attn_dropout) for _ in range(n_layers))
 
     def forward(self, tokens, lengths=None, readout: str = "tokens"):
         B, n, D = tokens.shape
