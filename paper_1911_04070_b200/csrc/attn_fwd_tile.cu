@@ -23,13 +23,13 @@ constexpr float kLn2 = 0.6931471805599453f;
 constexpr int kMaxKvRows = 208;  // staged K / V rows per chunk at k = 64 (union range + alignment slack)
 constexpr int kMaxRelRows = 80;  // staged relation rows per chunk (k + 1 <= 65, padded to 16)
 
-// Buffer sizes follow k, so that small k leaves room for more CTAs per SM and for a second set of
-// K / V / R buffers: with two sets the next chunk's rows are fetched while this chunk is computed.
+// Buffer sizes follow k, so that small k leaves room for more CTAs per SM.  (A second set of K / V / R
+// buffers, with the next chunk fetched while this one is computed, was measured at k = 4 and 8: 0.178 /
+// 0.377 ms against 0.151 / 0.306 ms for one set and the higher occupancy it allows.)
 struct FwdTileCfg {
     int kv_rows;    // K / V rows per buffer (multiple of 16)
     int rel_rows;   // relation rows per buffer (multiple of 16)
     int qr_stride;  // floats per row of the per-warp Q R^T scratch
-    int nbuf;       // 1 or 2 buffer sets
     int q_off, k_off, v_off, r_off, qr_off, bnd_off;  // byte offsets in shared memory
     size_t bytes;
 };
@@ -40,17 +40,11 @@ FwdTileCfg make_fwd_tile_cfg(const TreeParams& t, int chunks) {
     c.rel_rows = min(kMaxRelRows, (t.k + 1 + 15) & ~15);
     c.qr_stride = c.rel_rows - 4;                      // even, >= k + 1, not a multiple of 32 floats (bank spread)
     if (c.qr_stride < t.k + 1) c.qr_stride = c.rel_rows + 4;
-    const int per_set = 2 * c.kv_rows * 128 + c.rel_rows * 128;
-    const int rest = kTileTokens * 128 + 4 * 16 * c.qr_stride * 4 + chunks * (kTileTokens * 8 + 8);
-    // Measured at k = 4 and 8: one buffer set and more CTAs per SM (0.151 / 0.306 ms) beats two sets with the next
-    // chunk fetched under the current one (0.178 / 0.377 ms), so the second set stays off.
-    c.nbuf = 1;
-    (void)rest; (void)per_set;
     c.q_off = 0;
     c.k_off = kTileTokens * 128;
-    c.v_off = c.k_off + c.nbuf * c.kv_rows * 128;
-    c.r_off = c.v_off + c.nbuf * c.kv_rows * 128;
-    c.qr_off = c.r_off + c.nbuf * c.rel_rows * 128;
+    c.v_off = c.k_off + c.kv_rows * 128;
+    c.r_off = c.v_off + c.kv_rows * 128;
+    c.qr_off = c.r_off + c.rel_rows * 128;
     c.bnd_off = c.qr_off + 4 * 16 * c.qr_stride * 4;
     c.bytes = (size_t)c.bnd_off + (size_t)chunks * (kTileTokens * 8 + 8);
     return c;
@@ -71,7 +65,7 @@ fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
                 const int32_t* __restrict__ lengths, DropoutParams drop) {
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* q_s = smem + cfg.q_off;
-    unsigned char* k_s = smem + cfg.k_off;   // buffer set 0; set 1 follows at + kv_rows * 128 (K, V) / + rel_rows * 128 (R)
+    unsigned char* k_s = smem + cfg.k_off;
     unsigned char* v_s = smem + cfg.v_off;
     unsigned char* r_s = smem + cfg.r_off;
     float* qr_s = reinterpret_cast<float*>(smem + cfg.qr_off);
@@ -157,56 +151,47 @@ fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
     const int kQrStride = cfg.qr_stride;
     float* qr_w = qr_s + w * 16 * kQrStride;
     const int W = t.k + 1;
-    const uint32_t kv_set = (uint32_t)cfg.kv_rows * 128, r_set = (uint32_t)cfg.rel_rows * 128;
 
     auto next_chunk = [&](int c) {  // next chunk this tile reaches
         int cn = c + 1;
         while (cn < chunks && crange[cn].x > crange[cn].y) ++cn;
         return cn;
     };
-    // K / V rows of the chunk's node range and its relation rows -> buffer set `buf` (async)
-    auto stage = [&](int c, int buf) {
+    // K / V rows of the chunk's node range and its relation rows -> shared memory (async)
+    auto stage = [&](int c) {
         const int2 cr = crange[c];
         const int side = c >= n_left, level = side ? c - n_left : c;
         const int n_l = t.n >> level, id_base = node_id(t.n, level, 0);
         const int rel_base = side ? rel_right(t, level, 0) : rel_left(t, level, 0);
         const int base = cr.x & ~15;
         const int nr = min(cfg.kv_rows, (cr.y - base + 1 + 31 + 15) & ~15);
-        const uint32_t kb_u = k_u + buf * kv_set, vb_u = v_u + buf * kv_set, rb_u = r_u + buf * r_set;
         for (int idx = tid; idx < nr * 8; idx += 128) {
             const int row = idx >> 3, ch = idx & 7;
             const int node = min(base + row, n_l - 1);
             const size_t src = boff + (size_t)(id_base + node) * rs + ch * 8;
-            cp_async16(kb_u + tile_off(row, ch), k + src);
-            cp_async16(vb_u + tile_off(row, ch), v + src);
+            cp_async16(k_u + tile_off(row, ch), k + src);
+            cp_async16(v_u + tile_off(row, ch), v + src);
         }
         for (int idx = tid; idx < cfg.rel_rows * 8; idx += 128) {
             const int row = idx >> 3, ch = idx & 7;
-            if (row < W) cp_async16(rb_u + tile_off(row, ch), r + (size_t)(rel_base + row) * 64 + ch * 8);
-            else *reinterpret_cast<uint4*>(r_s + buf * r_set + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
+            if (row < W) cp_async16(r_u + tile_off(row, ch), r + (size_t)(rel_base + row) * 64 + ch * 8);
+            else *reinterpret_cast<uint4*>(r_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
         }
         cp_async_commit();
     };
 
-    __syncthreads();  // the prologue's reads of buffer set 0 are done; crange (and the masked ranges) are visible
-    int c = next_chunk(-1), it = 0;
-    if (c < chunks) stage(c, 0);
+    __syncthreads();  // the prologue's reads of the K / V / R buffers are done; crange (and the masked ranges) are visible
+    int c = next_chunk(-1);
+    if (c < chunks) stage(c);
     while (c < chunks) {
         const int cn = next_chunk(c);
-        const int buf = cfg.nbuf == 2 ? (it & 1) : 0;
-        if (cfg.nbuf == 2 && cn < chunks) {  // fetch the next chunk into the other set while this one is computed
-            stage(cn, buf ^ 1);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
+        cp_async_wait<0>();
         __syncthreads();  // this chunk's rows are in place
         const int2 cr = crange[c];
         const int side = c >= n_left;
         const int level = side ? c - n_left : c;
         const int id_base = node_id(t.n, level, 0);
         const int base = cr.x & ~15;
-        const uint32_t k_u = smem_u32(k_s) + buf * kv_set, v_u = smem_u32(v_s) + buf * kv_set, r_u = smem_u32(r_s) + buf * r_set;
 
         const int2* bc = bnd + c * kTileTokens;
         const int2 wr = rows_union(bc, r0, 16, lane);
@@ -314,10 +299,9 @@ fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
             }
         }
         }
-        __syncthreads();  // everyone is done with this buffer set
-        if (cfg.nbuf == 1 && cn < chunks) stage(cn, 0);
+        __syncthreads();  // everyone is done with the buffers
+        if (cn < chunks) stage(cn);
         c = cn;
-        ++it;
     }
 
     // ---- epilogue: normalise, round once to bf16, coalesced stores through the Q tile -----
