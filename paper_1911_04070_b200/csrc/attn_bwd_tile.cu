@@ -42,7 +42,8 @@ constexpr int kDrelGroups = 32;   // first stage of the d_rel sum
 struct ChunkPlan {
     int n_left, n_right;
     int slab_row0[kMaxChunks + 1];  // first reserved partial row of each chunk; [chunks] = rows per tile
-    int rel_rows;                   // relation rows reserved per chunk in the d_rel partials (multiple of 16)
+    int rel_rows;                   // relation offsets a chunk's products cover (multiple of 16)
+    int rel_store;                  // rows kept per chunk in the d_rel partials: k + 2, the most a chunk uses
 };
 
 struct BwdTileSmem {
@@ -184,7 +185,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
 
     float* qr_w = qr_s + rg * 16 * kQrStride;
     float* slab_cta = slabs + ((size_t)blockIdx.y * tiles + tile) * plan.slab_row0[chunks] * 128;
-    float* drel_cta = drel_part + ((size_t)blockIdx.y * tiles + tile) * chunks * plan.rel_rows * 64;
+    float* drel_cta = drel_part + ((size_t)blockIdx.y * tiles + tile) * chunks * plan.rel_store * 64;
 
     // K / V rows of the chunk's node range and its relation rows -> shared memory (async)
     auto stage = [&](int c) {
@@ -349,8 +350,8 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
         // next chunk that this tile reaches: its K / V / R rows arrive while phase 2 runs
         int cn = c + 1;
         while (cn < chunks && crange[cn].x > crange[cn].y) {  // a level no token of the tile reaches: zero d_rel partial
-            float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)cn * plan.rel_rows * 64);
-            for (int idx = tid; idx < plan.rel_rows * 16; idx += kBwdThreads) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+            float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)cn * plan.rel_store * 64);
+            for (int idx = tid; idx < plan.rel_store * 16; idx += kBwdThreads) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
             ++cn;
         }
         if (cn < chunks) stage(cn);
@@ -417,10 +418,12 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const int o = ot * 16 + g + hh * 8;
-                    float* dst = drel_cta + ((size_t)c * plan.rel_rows + o) * 64 + hc * 32 + c2;
+                    if (o < plan.rel_store) {
+                        float* dst = drel_cta + ((size_t)c * plan.rel_store + o) * 64 + hc * 32 + c2;
 #pragma unroll
-                    for (int nt = 0; nt < 4; ++nt)
-                        *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ar[nt][hh * 2], ar[nt][hh * 2 + 1]);
+                        for (int nt = 0; nt < 4; ++nt)
+                            *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ar[nt][hh * 2], ar[nt][hh * 2 + 1]);
+                    }
                 }
             }
         }
@@ -535,7 +538,7 @@ __global__ void drel_final_kernel(TreeParams t, ChunkPlan plan, const float* __r
     else if (rid < 1 + 2 * t.L * W) { const int j = (rid - 1 - t.L * W) / W; if (j < plan.n_right) { c = plan.n_left + j; off = (rid - 1 - t.L * W) % W; } }
     float acc = 0.f;
     if (c >= 0) {
-        const size_t at = ((size_t)c * plan.rel_rows + off) * 64 + ch;
+        const size_t at = ((size_t)c * plan.rel_store + off) * 64 + ch;
         for (int gi = 0; gi < kDrelGroups; ++gi) acc += grp[(size_t)gi * per_cta + at];
     }
     d_rel[x] = accumulate ? d_rel[x] + acc * scale : acc * scale;
@@ -563,12 +566,13 @@ ChunkPlan make_plan(const TreeParams& t) {
     }
     p.slab_row0[p.n_left + p.n_right] = at;
     p.rel_rows = (t.k + 2 + 15) & ~15;
+    p.rel_store = t.k + 2;
     return p;
 }
 
 TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, int B, int H, void* base) {
     const int chunks = plan.n_left + plan.n_right, tiles = t.n / kTileTokens;
-    const size_t per_pair = ((size_t)tiles * ((size_t)plan.slab_row0[chunks] * 128 + (size_t)chunks * plan.rel_rows * 64) +
+    const size_t per_pair = ((size_t)tiles * ((size_t)plan.slab_row0[chunks] * 128 + (size_t)chunks * plan.rel_store * 64) +
                              bwd_span_slab_floats(t, 1) + bwd_span_ext_floats(t, 1)) * sizeof(float);
     TileWorkspace w;
     size_t pairs = kPassBytes / per_pair;
@@ -581,8 +585,8 @@ TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, int B, int 
     w.aff_slab = (float*)(c + off); off += align256(sizeof(float) * bwd_span_slab_floats(t, (int)pairs));
     w.ext_dq = (float*)(c + off); off += align256(sizeof(float) * bwd_span_ext_floats(t, (int)pairs));
     w.slabs = (float*)(c + off); off += align256(sizeof(float) * pairs * tiles * plan.slab_row0[chunks] * 128);
-    w.drel_part = (float*)(c + off); off += align256(sizeof(float) * pairs * tiles * chunks * plan.rel_rows * 64);
-    w.drel_grp = (float*)(c + off); off += align256(sizeof(float) * kDrelGroups * chunks * plan.rel_rows * 64);
+    w.drel_part = (float*)(c + off); off += align256(sizeof(float) * pairs * tiles * chunks * plan.rel_store * 64);
+    w.drel_grp = (float*)(c + off); off += align256(sizeof(float) * kDrelGroups * chunks * plan.rel_store * 64);
     w.bytes = off;
     return w;
 }
@@ -611,7 +615,7 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
         return BPT_ERR_CUDA;
 
     const int total = p.B * p.H;
-    const size_t per_cta = (size_t)chunks * plan.rel_rows * 64;
+    const size_t per_cta = (size_t)chunks * plan.rel_store * 64;
     for (int pair0 = 0; pair0 < total; pair0 += ws.pairs_per_pass) {
         const int np = min(ws.pairs_per_pass, total - pair0);
         if (np > 65535) return BPT_ERR_UNSUPPORTED;

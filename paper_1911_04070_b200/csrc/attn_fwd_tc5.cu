@@ -4,9 +4,10 @@
 //
 // One CTA = 128 consecutive tokens of one (batch entry, head) = the 128 lanes of tensor memory,
 // four threads per token row (warps w, w + 4, w + 8, w + 12 read the same lane quadrant), each
-// taking a quarter of the columns, plus a driver warp.  Per (side, level) chunk the union node range of the tile (at most
-// 128 / 2^level + k + 2 nodes) is staged once in shared memory, and one elected thread issues
-//     QR = Q R_chunk^T   (128 x 80)        -- the relative-position terms of every offset
+// taking a quarter of the columns, plus a driver warp.  Per (side, level) chunk the union node range
+// of the tile (at most 128 / 2^level + k + 2 nodes) is staged once in shared memory, and one elected
+// thread issues
+//     QR = Q R_chunk^T   (128 x round16(k + 2)) -- the relative-position terms of every offset
 //     S  = Q K_range^T   (128 x N, N <= 208)
 // into tensor memory.  The row's bias values go to a shared table indexed [offset][row], so that
 // the per-row shift between node index and offset is plain address arithmetic; the part of S that
@@ -17,14 +18,15 @@
 // which each thread adds (its 16 channels) to the running output row with the usual rescale.
 // The self loop is offset 0 of the level-0 left chunk, as in the tiled backward.
 //
-// Warp roles: eight softmax warps and one driver warp.  The driver's elected thread brings the K, V and R
-// rows in with TMA (cp.async.bulk.tensor, 16-row boxes straight into the swizzled layout the
+// Warp roles: sixteen softmax warps and one driver warp.  The driver's elected thread brings the K, V
+// and R rows in with TMA (cp.async.bulk.tensor, 16-row boxes straight into the swizzled layout the
 // tensor core reads) and issues every MMA; mbarriers carry all hand-offs (rows landed -> driver,
-// S / QR done and O_chunk done -> softmax threads, P complete -> driver), so the softmax code has
-// no block-wide barrier.  QR and S of the next chunk are issued as soon as P of this one is
-// complete, the next K / R rows are fetched as soon as S is done (single buffers) and the next V
-// rows into the other of two buffers; O_chunk is collected at the start of the next chunk.
-// Every mbarrier wait gives up after about a second and the kernel then winds down.
+// S / QR done and O_chunk done -> softmax threads, scores read and P complete -> driver), so the
+// softmax code has no block-wide barrier.  QR and S of the next chunk are issued as soon as every
+// thread holds its part of this chunk's scores, the next K / R rows are fetched as soon as S is done
+// (single buffers) and the next V rows into the other of two buffers; O_chunk is collected just
+// before the next chunk's P is written.  Every mbarrier wait gives up after about a second and the
+// kernel then winds down.
 #include <cuda.h>
 
 #include "bpt_internal.cuh"
@@ -56,7 +58,7 @@ struct FwdTcSmem {
     static constexpr int p_off = r_off + kTcRelRows * 128;               // 4 key blocks of [128 rows][128 B]
     static constexpr int bias_off = p_off + 4 * kTcTokens * 128;         // [68 offsets][128 rows] fp32
     static constexpr int misc_off = bias_off + kTcBiasRows * kTcTokens * 4;  // 7 mbarriers, tensor-memory slot, abort flag
-    static constexpr int xch_off = misc_off + 64;                        // [2 halves][128 rows] fp32 exchange + the same of give-up flags
+    static constexpr int xch_off = misc_off + 64;                        // [kTpr][128 rows] fp32 exchange + the same of give-up flags
     static constexpr int bnd_off = xch_off + 2 * kTpr * kTcTokens * 4;          // [chunks][128] short2, then [chunks] int2
     static size_t bytes(int chunks) { return (size_t)bnd_off + (size_t)chunks * (kTcTokens * 4 + 8) + 1024; }
 };
