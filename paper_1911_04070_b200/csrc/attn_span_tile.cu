@@ -262,24 +262,25 @@ fwd_span_merge_kernel(TreeParams t, const float* __restrict__ ext_part, __nv_bfl
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (mx == -INFINITY) mx = 0.f;  // a span without real tokens: every partial is empty (2^-inf = 0 below)
-    // tiles in groups of 32: lane j owns the weight of tile 32 i + j, every lane adds its two channels of
-    // all tiles in tile order (the loads of a group do not depend on one another)
+    // tiles sixteen at a time: all loads of a batch are issued before any of them is used; summed in tile order
     float l = 0.f, a0 = 0.f, a1 = 0.f;
-    for (int x0 = 0; x0 < nT; x0 += 32) {
-        float f_mine = 0.f, l_mine = 0.f;
-        if (x0 + lane < nT) {
-            const float* p = base + (size_t)(x0 + lane) * stride;
-            f_mine = fast_exp2(p[0] - mx);
-            l_mine = p[1] * f_mine;
+    for (int x0 = 0; x0 < nT; x0 += 16) {
+        float mm[16], ll[16];
+        float2 aa[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+            const bool in = x0 + u < nT;
+            const float* p = base + (size_t)(in ? x0 + u : 0) * stride;
+            mm[u] = in ? p[0] : -INFINITY;
+            ll[u] = p[1];
+            aa[u] = *reinterpret_cast<const float2*>(p + 2 + lane * 2);
         }
-        const int cnt = min(32, nT - x0);
-#pragma unroll 8
-        for (int jj = 0; jj < cnt; ++jj) {
-            const float f = __shfl_sync(0xffffffffu, f_mine, jj);
-            const float2 a = *reinterpret_cast<const float2*>(base + (size_t)(x0 + jj) * stride + 2 + lane * 2);
-            l += __shfl_sync(0xffffffffu, l_mine, jj);
-            a0 = fmaf(a.x, f, a0);
-            a1 = fmaf(a.y, f, a1);
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+            const float f = fast_exp2(mm[u] - mx);  // 0 for the slots past the last tile
+            l = fmaf(ll[u], f, l);
+            a0 = fmaf(aa[u].x, f, a0);
+            a1 = fmaf(aa[u].y, f, a1);
         }
     }
     const float inv = l > 0.f ? 1.f / l : 0.f;  // l = 0: a span without real tokens
