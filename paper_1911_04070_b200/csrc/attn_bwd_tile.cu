@@ -31,11 +31,8 @@ bpt_status launch_bwd_span(const AttnProblem& p, int pair0, int n_pairs, float* 
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kKvRows = 208;      // staged K / V rows per chunk
-constexpr int kRelRows = 80;      // staged relation rows per chunk (k + 2 <= 66, padded to 16)
-constexpr int kQrStride = 76;     // floats per row of the per-warp Q R^T scratch
-constexpr int kPStride = 432;     // bytes per token row of the P / dS tiles (208 bf16 + 16: odd number of 16-byte chunks)
-constexpr int kSkewStride = 176;  // bytes per token row of the skewed dS tile (80 bf16 + 16)
+constexpr int kMaxKvRows = 208;   // staged K / V rows per chunk at k = 64
+constexpr int kMaxRelRows = 80;   // staged relation rows per chunk (k + 2 <= 66, padded to 16)
 constexpr int kMaxChunks = 2 * kMaxLevels;
 constexpr int kDrelGroups = 32;   // first stage of the d_rel sum
 
@@ -46,19 +43,49 @@ struct ChunkPlan {
     int rel_store;                  // rows kept per chunk in the d_rel partials: k + 2, the most a chunk uses
 };
 
-struct BwdTileSmem {
-    static constexpr int q_bytes = kTileTokens * 128;
-    static constexpr int kv_bytes = kKvRows * 128;
-    static constexpr int r_bytes = kRelRows * 128;
-    static constexpr int qr_bytes = 4 * 16 * kQrStride * 4;
-    static constexpr int p_bytes = kTileTokens * kPStride;
-    static constexpr int skew_bytes = kTileTokens * kSkewStride;
-    static constexpr int row_bytes = 2 * kTileTokens * 4;  // lse, delta
-    static constexpr int fixed = 2 * q_bytes + 2 * kv_bytes + r_bytes + qr_bytes + 2 * p_bytes + skew_bytes + row_bytes;
-    static size_t bytes(int chunks) { return (size_t)fixed + (size_t)chunks * (kTileTokens * 8 + 8); }
+// Shared-memory layout; the buffer sizes follow k.  Where two CTAs fit an SM the kernel runs with four
+// warps per CTA (one per group of 16 query rows), otherwise with eight (two per group).
+struct BwdTileCfg {
+    int kv_rows;      // staged K / V rows (multiple of 16)
+    int rel_rows;     // staged relation rows (multiple of 16)
+    int qr_stride;    // floats per row of the Q R^T scratch
+    int p_stride;     // bytes per token row of the P / dS tiles (an odd number of 16-byte chunks)
+    int skew_stride;  // bytes per token row of the skewed dS tile (an odd number of 16-byte chunks)
+    int g_off, k_off, v_off, r_off, qr_off, p_off, ds_off, sk_off, row_off, bnd_off;  // byte offsets (Q tile at 0)
+    size_t bytes;
 };
 
-constexpr int kBwdThreads = 256;  // 8 warps: two per group of 16 query rows
+constexpr BwdTileCfg layout_of(int kv_rows, int rel_rows, int qr_stride) {
+    BwdTileCfg c{};
+    c.kv_rows = kv_rows;
+    c.rel_rows = rel_rows;
+    c.qr_stride = qr_stride;
+    c.p_stride = kv_rows * 2 + 16;
+    c.skew_stride = rel_rows * 2 + 16;
+    c.g_off = kTileTokens * 128;
+    c.k_off = c.g_off + kTileTokens * 128;
+    c.v_off = c.k_off + kv_rows * 128;
+    c.r_off = c.v_off + kv_rows * 128;
+    c.qr_off = c.r_off + rel_rows * 128;
+    c.p_off = c.qr_off + 4 * 16 * qr_stride * 4;
+    c.ds_off = c.p_off + kTileTokens * c.p_stride;
+    c.sk_off = c.ds_off + kTileTokens * c.p_stride;
+    c.row_off = c.sk_off + kTileTokens * c.skew_stride;
+    c.bnd_off = c.row_off + 2 * kTileTokens * 4;
+    return c;
+}
+// the sizes of k = 64: the eight-warp kernel has this layout as compile-time constants
+constexpr BwdTileCfg kWidestCfg = layout_of(kMaxKvRows, kMaxRelRows, kMaxRelRows - 4);
+
+BwdTileCfg make_bwd_tile_cfg(const TreeParams& t, int chunks, bool widest) {
+    BwdTileCfg c = kWidestCfg;
+    if (!widest) {
+        const int rel_rows = min(kMaxRelRows, (t.k + 2 + 15) & ~15);
+        c = layout_of(min(kMaxKvRows, (t.kc + 143) & ~15), rel_rows, rel_rows - 4 >= t.k + 2 ? rel_rows - 4 : rel_rows + 4);
+    }
+    c.bytes = (size_t)c.bnd_off + (size_t)chunks * (kTileTokens * 8 + 8);
+    return c;
+}
 
 // barrier of the two warps that share a group of query rows (ids 1..4; id 0 is __syncthreads)
 __device__ __forceinline__ void pair_barrier(int rg) {
@@ -84,12 +111,13 @@ __device__ __forceinline__ ChunkGeom chunk_geom(const TreeParams& t, int n_left,
     gm.n_rel_c = c == 0 ? t.k + 2 : t.k + 1;  // chunk 0 also holds r^self
     gm.base = cr.x & ~15;
     gm.kend = cr.y - gm.base;
-    gm.nr = min(kKvRows, (gm.kend + 1 + 31 + 15) & ~15);
+    gm.nr = (gm.kend + 1 + 31 + 15) & ~15;  // capped by the caller's buffer
     return gm;
 }
 
-__global__ void __launch_bounds__(kBwdThreads)
-bwd_tile_kernel(TreeParams t, ChunkPlan plan,
+template <int NW>  // warps per CTA: 8 (two per group of 16 query rows) or 4 (one per group)
+__global__ void __launch_bounds__(NW * 32)
+bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
                 const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                 const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
                 const __nv_bfloat16* __restrict__ out, const float* __restrict__ lse,
@@ -97,23 +125,27 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 int2* __restrict__ tile_range, float* __restrict__ slabs, float* __restrict__ drel_part,
                 int H, int pair0, float scale, const int32_t* __restrict__ lengths, DropoutParams drop) {
     extern __shared__ __align__(128) unsigned char smem[];
+    const BwdTileCfg cfg = NW == 8 ? kWidestCfg : cfg_arg;  // eight warps: the widest layout, all constants
     unsigned char* q_s = smem;
-    unsigned char* g_s = q_s + BwdTileSmem::q_bytes;   // d_out tile
-    unsigned char* k_s = g_s + BwdTileSmem::q_bytes;
-    unsigned char* v_s = k_s + BwdTileSmem::kv_bytes;
-    unsigned char* r_s = v_s + BwdTileSmem::kv_bytes;
-    float* qr_s = reinterpret_cast<float*>(r_s + BwdTileSmem::r_bytes);
-    unsigned char* p_s = reinterpret_cast<unsigned char*>(qr_s) + BwdTileSmem::qr_bytes;
-    unsigned char* ds_s = p_s + BwdTileSmem::p_bytes;
-    unsigned char* sk_s = ds_s + BwdTileSmem::p_bytes;
-    float* lse_s = reinterpret_cast<float*>(sk_s + BwdTileSmem::skew_bytes);
+    unsigned char* g_s = smem + cfg.g_off;   // d_out tile
+    unsigned char* k_s = smem + cfg.k_off;
+    unsigned char* v_s = smem + cfg.v_off;
+    unsigned char* r_s = smem + cfg.r_off;
+    float* qr_s = reinterpret_cast<float*>(smem + cfg.qr_off);
+    unsigned char* p_s = smem + cfg.p_off;
+    unsigned char* ds_s = smem + cfg.ds_off;
+    unsigned char* sk_s = smem + cfg.sk_off;
+    float* lse_s = reinterpret_cast<float*>(smem + cfg.row_off);
     float* delta_s = lse_s + kTileTokens;
     int2* bnd = reinterpret_cast<int2*>(delta_s + kTileTokens);
     const int n_left = plan.n_left, n_right = plan.n_right, chunks = n_left + n_right;
     int2* crange = bnd + chunks * kTileTokens;
 
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int rg = w & 3, half = w >> 2;  // row group (16 query rows) and which of its two warps
+    constexpr int kBwdThreads = NW * 32;
+    constexpr bool kPair = NW == 8;
+    const int kQrStride = cfg.qr_stride, kPStride = cfg.p_stride, kSkewStride = cfg.skew_stride;
+    const int rg = w & 3, half = kPair ? w >> 2 : 0;  // row group (16 query rows) and, with eight warps, which of its two warps
     const int g = lane >> 2, c2 = (lane & 3) * 2;
     const int tile = blockIdx.x, tiles = gridDim.x, t0 = tile * kTileTokens;
     const int pair = pair0 + blockIdx.y, b = pair / H, h = pair % H;
@@ -190,14 +222,15 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
     // K / V rows of the chunk's node range and its relation rows -> shared memory (async)
     auto stage = [&](int c) {
         const ChunkGeom gm = chunk_geom(t, n_left, c, crange[c]);
-        for (int idx = tid; idx < gm.nr * 8; idx += kBwdThreads) {
+        const int nr = min(cfg.kv_rows, gm.nr);
+        for (int idx = tid; idx < nr * 8; idx += kBwdThreads) {
             const int row = idx >> 3, ch = idx & 7;
             const int node = min(gm.base + row, gm.n_l - 1);
             const size_t src = boff + (size_t)(gm.id_base + node) * rs + ch * 8;
             cp_async16(k_u + tile_off(row, ch), k + src);
             cp_async16(v_u + tile_off(row, ch), v + src);
         }
-        for (int idx = tid; idx < kRelRows * 8; idx += kBwdThreads) {
+        for (int idx = tid; idx < cfg.rel_rows * 8; idx += kBwdThreads) {
             const int row = idx >> 3, ch = idx & 7;
             if (row < gm.n_rel_c) cp_async16(r_u + tile_off(row, ch), r + (size_t)(gm.rel_base + row) * 64 + ch * 8);
             else *reinterpret_cast<uint4*>(r_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
@@ -229,8 +262,8 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
         const bool w_any = wr.x <= wr.y;
         if (w_any) {  // Q R^T for the chunk's relation rows -> the row group's scratch
 #pragma unroll
-            for (int np = 0; np < kRelRows / 16; ++np) {
-                if (np * 16 < n_rel_c && (np & 1) == half) {
+            for (int np = 0; np < kMaxRelRows / 16; ++np) {
+                if (np * 16 < n_rel_c && (!kPair || (np & 1) == half)) {
                     float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
@@ -250,16 +283,15 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 }
             }
         }
-        pair_barrier(rg);
+        if constexpr (kPair) pair_barrier(rg); else __syncwarp();
 
         const int2 ba = bc[r0 + g], bb = bc[r0 + g + 8];
         const int lo_r[2] = {ba.x, bb.x}, hi_r[2] = {ba.y, bb.y};
         const float lse_r[2] = {lse_s[r0 + g], lse_s[r0 + g + 8]};
         const float del_r[2] = {delta_s[r0 + g], delta_s[r0 + g + 8]};
         const int w_lo = w_any ? wr.x - base : 1 << 30, w_hi = w_any ? wr.y - base : -1;
-        // every 32-key block is shared: this warp takes 16 of its keys (balanced whatever the block count)
-        for (int kb0 = 0; kb0 <= kend; kb0 += 32) {
-            const int kb = kb0 + half * 16;
+        // 16 keys of a block: S, dP, the element-wise part, P / dS / skew to shared memory, dQ += dS K
+        auto keys16 = [&](int kb) {
             unsigned char* p_row0 = p_s + (r0 + g) * kPStride + (kb + c2) * 2;
             unsigned char* d_row0 = ds_s + (r0 + g) * kPStride + (kb + c2) * 2;
             if (kb + 15 < w_lo || kb > w_hi) {  // nothing of these rows here: zeros for phase 2
@@ -270,7 +302,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                     *reinterpret_cast<uint32_t*>(d_row0 + j * 16) = 0u;
                     *reinterpret_cast<uint32_t*>(d_row0 + 8 * kPStride + j * 16) = 0u;
                 }
-                continue;
+                return;
             }
             float s[2][4], dp[2][4];
 #pragma unroll
@@ -327,12 +359,21 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
                 mma_bf16(acc_q[np * 2], da, bf[0], bf[1]);
                 mma_bf16(acc_q[np * 2 + 1], da, bf[2], bf[3]);
             }
+        };
+        // with eight warps every 32-key block is shared: this warp takes 16 of its keys (balanced whatever the block count)
+        for (int kb0 = 0; kb0 <= kend; kb0 += 32) {
+            if constexpr (kPair) {
+                keys16(kb0 + half * 16);
+            } else {
+                keys16(kb0);
+                keys16(kb0 + 16);
+            }
         }
-        pair_barrier(rg);  // the group's rows of the skew tile are complete
+        if constexpr (kPair) pair_barrier(rg); else __syncwarp();  // the group's rows of the skew tile are complete
         if (w_any) {       // dQ += skew(dS) R_chunk, the k-steps shared out between the two warps
 #pragma unroll
-            for (int kk = 0; kk < kRelRows / 16; ++kk) {
-                if (kk * 16 < n_rel_c && (kk & 1) == half) {
+            for (int kk = 0; kk < kMaxRelRows / 16; ++kk) {
+                if (kk * 16 < n_rel_c && (!kPair || (kk & 1) == half)) {
                     uint32_t a[4];
                     load_a_plain(sk_u, kSkewStride, r0, kk * 16, lane, a);
 #pragma unroll
@@ -434,7 +475,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
     // ---- epilogue: the two warps' dq parts are added (second warp's part through shared memory), ----
     // ---- dq = scale * sum, rounded once to bf16, coalesced stores through the Q tile              ----
     float* red = reinterpret_cast<float*>(p_s) + rg * 16 * 64;  // [16 rows][64] per row group
-    if (half == 1) {
+    if (kPair && half == 1) {
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
             *reinterpret_cast<float2*>(red + g * 64 + nt * 8 + c2) = make_float2(acc_q[nt][0], acc_q[nt][1]);
@@ -445,8 +486,8 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan,
     if (half == 0) {
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
-            const float2 x = *reinterpret_cast<const float2*>(red + g * 64 + nt * 8 + c2);
-            const float2 y = *reinterpret_cast<const float2*>(red + (g + 8) * 64 + nt * 8 + c2);
+            const float2 x = kPair ? *reinterpret_cast<const float2*>(red + g * 64 + nt * 8 + c2) : make_float2(0.f, 0.f);
+            const float2 y = kPair ? *reinterpret_cast<const float2*>(red + (g + 8) * 64 + nt * 8 + c2) : make_float2(0.f, 0.f);
             *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g, nt) + c2 * 2) =
                 pack_bf16((acc_q[nt][0] + x.x) * scale, (acc_q[nt][1] + x.y) * scale);
             *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g + 8, nt) + c2 * 2) =
@@ -609,9 +650,13 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
     const ChunkPlan plan = make_plan(t);
     const int chunks = plan.n_left + plan.n_right, tiles = t.n / kTileTokens, N = 2 * t.n - 1;
     const TileWorkspace ws = carve_tile(t, plan, p.B, p.H, p.workspace);
-    const size_t smem = BwdTileSmem::bytes(chunks);
+    BwdTileCfg cfg = make_bwd_tile_cfg(t, chunks, false);
+    const bool four = cfg.bytes <= 112 * 1024;  // two CTAs fit an SM: four warps each, independent barriers
+    if (!four) cfg = make_bwd_tile_cfg(t, chunks, true);
+    const size_t smem = cfg.bytes;
     if (smem > 227 * 1024) return BPT_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(bwd_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    auto kernel = four ? bwd_tile_kernel<4> : bwd_tile_kernel<8>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return BPT_ERR_CUDA;
 
     const int total = p.B * p.H;
@@ -622,8 +667,8 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
         // span rows: dq of the spans and, per token, the affiliated edges' share of dk / dv
         const bpt_status s = launch_bwd_span(p, pair0, np, ws.ext_dq, ws.aff_slab);
         if (s != BPT_OK) return s;
-        bwd_tile_kernel<<<dim3(tiles, np), kBwdThreads, smem, p.stream>>>(
-            t, plan, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
+        kernel<<<dim3(tiles, np), four ? 128 : 256, smem, p.stream>>>(
+            t, plan, cfg, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
             (const __nv_bfloat16*)p.rel_emb, (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out,
             (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale, p.lengths, p.drop);
         trace_mark(p.stream, "bwd_tile");
