@@ -34,7 +34,7 @@ typedef enum {
     BPT_ERR_UNSUPPORTED = 2,  /* head size / dtype / range the kernels do not cover        */
     BPT_ERR_WORKSPACE = 3,    /* workspace missing or smaller than the size query says      */
     BPT_ERR_CUDA = 4,         /* a CUDA runtime call or launch failed                       */
-    BPT_ERR_TIMEOUT = 5,      /* reserved: a bounded device-side wait expired               */
+    BPT_ERR_TIMEOUT = 5,      /* a bounded device-side wait expired (see bpt_attn_fwd)      */
     BPT_ERR_OVERFLOW = 6,     /* edge count does not fit the 32-bit index arrays            */
     BPT_ERR_SCRATCH_LIMIT = 7 /* problem needs more scratch than the built-in static array  */
 } bpt_status;
@@ -114,6 +114,11 @@ size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_
  * `scale` is explicit (the paper divides by sqrt(d); callers pass 1/sqrt(d)).
  * d must be 32 or 64.  `g` is a host pointer to a struct of device pointers.
  * `workspace` may be NULL when the size query returns 0.
+ * Device-side failure report: the kernels that wait on hardware barriers (tensor-memory forward)
+ * bound every wait to about a second; if one expires the kernel winds down, the results are
+ * invalid and BPT_ERR_TIMEOUT is stored in the 32-bit word at workspace + (size query) - 256,
+ * which the call never clears: zero it before the call if you want to read it afterwards
+ * (after synchronising the stream).
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
  */
 bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,

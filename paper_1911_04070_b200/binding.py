@@ -259,6 +259,15 @@ def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, work
     return dq, dk, dv, d_rel
 
 
+def bpt_forward_status(workspace) -> int:
+    """The device-side status word of a forward workspace (0 = ok, 5 = a bounded wait expired), read after a
+    stream synchronisation.  The library never clears it: zero the workspace before the call."""
+    if workspace is None or workspace.numel() < 256:
+        return 0
+    torch.cuda.synchronize(workspace.device)
+    return int(workspace[-256:-252].view(torch.int32).item())
+
+
 def bpt_static_scratch_bytes() -> int:
     return int(load_library().bpt_static_scratch_bytes())
 

@@ -26,10 +26,12 @@ for n, k, flags, B, H in cases:
     x = synth.make_inputs(B, ref.n_nodes, H, 64, ref.n_rel, seed=7 + n + k, std_qkv=0.5, std_rel=0.3, bf16=True, with_grad=False)
     g = binding.bpt_build_graph(n, k, flags, device="cuda:0", with_transpose=False)
     t = {a: torch.from_numpy(b).to("cuda:0", torch.bfloat16) for a, b in x.items()}
+    ws = torch.zeros(binding.bpt_attn_workspace_bytes(g, B, H, 64, binding.BPT_BF16, False), dtype=torch.uint8, device="cuda:0")
     binding.bpt_trace_begin(8)
-    out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125)
+    out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125, workspace=ws)
     names = [a for a, _ in binding.bpt_trace_end(8)]
     assert "fwd_tc5" in names, names          # the tensor-memory kernel really ran
+    assert binding.bpt_forward_status(ws) == 0   # no bounded wait gave up
     o_ref, lse_ref = ctwin.attn_fwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], 0.125)
     assert_close("out", out.float().cpu().numpy(), o_ref, TOL["bf16"])
     assert_close("lse", lse.cpu().numpy(), lse_ref, TOL["bf16"])
