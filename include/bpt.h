@@ -199,6 +199,20 @@ bpt_status bpt_attn_bwd_ex(const bpt_graph* g, int32_t B, int32_t H, int32_t d, 
                            void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Forward for a few destination rows only -- the building block of step-by-step decoding with the
+ * left-only graph (Sec. 4.2 uses BPT autoregressively): when token i arrives, the rows that change in
+ * a layer are token i and its L ancestors, and with lengths[b] = i + 1 the ancestors attend exactly
+ * the tokens seen so far.  rows: device array [B][n_rows] of node ids (one list per batch entry;
+ * ids outside [0, n_nodes) are skipped); only those rows of out and lse are written.  Same equation,
+ * options and layouts as bpt_attn_fwd_ex; runs on the general row kernel, needs no workspace.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+bpt_status bpt_attn_fwd_rows(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                             const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                             const bpt_attn_options* opt, const int32_t* rows, int32_t n_rows,
+                             void* out, float* lse, void* cuda_stream);
+
+/*
  * Backward pass for callers that must not allocate device memory (the paper has no
  * counterpart; this is a deployment convenience).
  *

@@ -20,7 +20,7 @@ BPT_F32, BPT_BF16 = 0, 1
 EXPORTS = ("bpt_graph_dims_query", "bpt_build_graph", "bpt_attn_workspace_bytes", "bpt_attn_fwd",
            "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end",
            "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch", "bpt_attn_fwd_varlen", "bpt_attn_bwd_varlen",
-           "bpt_attn_fwd_ex", "bpt_attn_bwd_ex")
+           "bpt_attn_fwd_ex", "bpt_attn_bwd_ex", "bpt_attn_fwd_rows")
 
 
 class BptError(RuntimeError):
@@ -81,6 +81,9 @@ def load_library() -> ctypes.CDLL:
         lib.bpt_attn_bwd_ex.restype = ctypes.c_int
         lib.bpt_attn_bwd_ex.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
                                         ctypes.POINTER(AttnOptions), vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.bpt_attn_fwd_rows.restype = ctypes.c_int
+        lib.bpt_attn_fwd_rows.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
+                                          ctypes.POINTER(AttnOptions), vp, i32, vp, vp, vp]
         lib.bpt_static_scratch_bytes.restype = sz
         lib.bpt_static_scratch_bytes.argtypes = []
         lib.bpt_attn_bwd_static_scratch.restype = ctypes.c_int
@@ -257,6 +260,25 @@ def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, work
                                            _ptr(dk), _ptr(dv), _ptr(d_rel), _ptr(workspace), ws_n, _stream()),
                    "bpt_attn_bwd_varlen")
     return dq, dk, dv, d_rel
+
+
+def bpt_attn_fwd_rows(g: Graph, q, k, v, rel_emb, scale: float, rows, out, lse, lengths=None,
+                      dropout_p: float = 0.0, dropout_seed: int = 0):
+    """Recomputes the listed destination rows of (out, lse) in place.  rows: int32 [B, n_rows] node ids on the
+    device (one list per batch entry).  The building block of step-by-step decoding: token i and its
+    ancestors, with lengths = i + 1."""
+    _check_layout(g, q, k, v, out)
+    B, N, H, d = q.shape
+    if rows.dtype != torch.int32 or rows.dim() != 2 or rows.shape[0] != B or not rows.is_contiguous() or rows.device != q.device:
+        raise ValueError("rows must be a contiguous int32 tensor [B, n_rows] on the device of q")
+    if lengths is not None:
+        _check_lengths(lengths, q)
+    opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed))
+    with torch.cuda.device(q.device):
+        _check(load_library().bpt_attn_fwd_rows(ctypes.byref(g.c), B, H, d, _dtype_code(q), _ptr(q), _ptr(k), _ptr(v),
+                                                _ptr(rel_emb), float(scale), ctypes.byref(opt), _ptr(rows), rows.shape[1],
+                                                _ptr(out), _ptr(lse), _stream()), "bpt_attn_fwd_rows")
+    return out, lse
 
 
 def bpt_forward_status(workspace) -> int:

@@ -21,6 +21,8 @@ extern "C" size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_
     return backward ? bwd_workspace_bytes(*g, B, H, d, dtype) : fwd_workspace_bytes(*g, B, H, d, dtype);
 }
 
+static bool options_ok(const bpt_attn_options* opt) { return !opt || (opt->dropout_p >= 0.f && opt->dropout_p < 1.f); }
+
 static bpt_status attn_fwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                 const void* q, const void* k, const void* v, const void* rel_emb, float scale,
                                 const int32_t* lengths, DropoutParams drop, void* out, float* lse, void* workspace,
@@ -55,8 +57,6 @@ extern "C" bpt_status bpt_attn_fwd_varlen(const bpt_graph* g, int32_t B, int32_t
     return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, make_dropout(0.f, 0), out, lse, workspace, workspace_bytes, cuda_stream);
 }
 
-static bool options_ok(const bpt_attn_options* opt) { return !opt || (opt->dropout_p >= 0.f && opt->dropout_p < 1.f); }
-
 extern "C" bpt_status bpt_attn_fwd_ex(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                       const void* q, const void* k, const void* v, const void* rel_emb, float scale,
                                       const bpt_attn_options* opt, void* out, float* lse, void* workspace,
@@ -87,6 +87,25 @@ static bpt_status attn_bwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_
     p.workspace = workspace; p.workspace_bytes = workspace_bytes;
     p.stream = (cudaStream_t)cuda_stream;
     return launch_bwd(p);
+}
+
+extern "C" bpt_status bpt_attn_fwd_rows(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
+                                        const void* q, const void* k, const void* v, const void* rel_emb, float scale,
+                                        const bpt_attn_options* opt, const int32_t* rows, int32_t n_rows,
+                                        void* out, float* lse, void* cuda_stream) {
+    const bpt_status s = check_problem(g, B, H, d, dtype, false);
+    if (s != BPT_OK) return s;
+    if (!q || !k || !v || !rel_emb || !out || !lse || !rows || n_rows < 1 || !options_ok(opt)) return BPT_ERR_INVALID_ARG;
+    AttnProblem p{};
+    p.g = g;
+    tree_params_from_dims(g->dims, &p.tree);
+    p.B = B; p.H = H; p.d = d; p.dtype = dtype;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale;
+    p.lengths = opt ? opt->lengths : nullptr;
+    p.drop = opt ? make_dropout(opt->dropout_p, opt->dropout_seed) : make_dropout(0.f, 0);
+    p.out = out; p.lse = lse;
+    p.stream = (cudaStream_t)cuda_stream;
+    return launch_fwd_row_list(p, rows, n_rows);
 }
 
 extern "C" bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,

@@ -18,15 +18,18 @@ __global__ void __launch_bounds__(256)
 fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col, const int32_t* __restrict__ rel,
                 const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
                 T* __restrict__ out, float* __restrict__ lse, int N, int row0, int nrows, int H, int ngroups,
-                float scale_log2e, const int32_t* __restrict__ lengths, DropoutParams drop) {
+                float scale_log2e, const int32_t* __restrict__ lengths, DropoutParams drop,
+                const int32_t* __restrict__ row_list) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
     const int nw = blockDim.x >> 5, w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t bid = blockIdx.x;
-    const int u = row0 + nrows - 1 - (int)(bid % nrows);  // rows [row0, row0 + nrows), long span rows first
+    // rows [row0, row0 + nrows), long span rows first; or the nrows rows of row_list (per batch entry: [B][nrows])
     const int hg = (int)((bid / nrows) % ngroups);
     const int b = (int)(bid / ((int64_t)nrows * ngroups));
+    const int u = row_list ? row_list[(size_t)b * nrows + (int)(bid % nrows)] : row0 + nrows - 1 - (int)(bid % nrows);
+    if (u < 0 || u >= N) return;  // an entry of row_list outside the graph is skipped (uniform over the CTA)
     const int head = hg * M::HPW + lane / M::G;
     const bool head_ok = head < H;
     const int hc = head_ok ? head : H - 1;
@@ -133,7 +136,7 @@ int rows_kernel_warps(const bpt_graph& g) {
 }
 
 template <typename T, int D>
-static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows) {
+static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows, const int32_t* row_list = nullptr) {
     using M = RowMap<T, D>;
     constexpr int U = 4;
     const bpt_graph& g = *p.g;
@@ -145,7 +148,7 @@ static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows) {
     const size_t smem = nw > 1 ? (size_t)nw * 32 * (2 + M::EPL) * sizeof(float) : 0;
     fwd_rows_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e, p.lengths, p.drop);
+        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e, p.lengths, p.drop, row_list);
     trace_mark(p.stream, "fwd_rows");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }
@@ -185,6 +188,12 @@ bpt_status launch_fwd(const AttnProblem& p) {
     const int row0 = 0, nrows = p.g->dims.n_nodes;
     if (p.dtype == BPT_F32) return p.d == 64 ? launch_rows<float, 64>(p, row0, nrows) : launch_rows<float, 32>(p, row0, nrows);
     return p.d == 64 ? launch_rows<__nv_bfloat16, 64>(p, row0, nrows) : launch_rows<__nv_bfloat16, 32>(p, row0, nrows);
+}
+
+// The listed destination rows only, through the general row kernel (any dtype / head size the library takes).
+bpt_status launch_fwd_row_list(const AttnProblem& p, const int32_t* rows, int n_rows) {
+    if (p.dtype == BPT_F32) return p.d == 64 ? launch_rows<float, 64>(p, 0, n_rows, rows) : launch_rows<float, 32>(p, 0, n_rows, rows);
+    return p.d == 64 ? launch_rows<__nv_bfloat16, 64>(p, 0, n_rows, rows) : launch_rows<__nv_bfloat16, 32>(p, 0, n_rows, rows);
 }
 
 }  // namespace bpt

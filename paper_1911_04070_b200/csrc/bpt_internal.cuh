@@ -41,6 +41,7 @@ void trace_mark(cudaStream_t st, const char* name);
 size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype);
 size_t bwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype);
 bpt_status launch_fwd(const AttnProblem& p);
+bpt_status launch_fwd_row_list(const AttnProblem& p, const int32_t* rows, int n_rows);
 bpt_status launch_bwd(const AttnProblem& p);
 
 }  // namespace bpt
