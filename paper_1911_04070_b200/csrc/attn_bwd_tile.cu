@@ -1,14 +1,14 @@
 // Tiled backward for the token rows (arXiv 1911.04070: gradient of the Sec. 3.4 equation over
 // the contextual edges of Sec. 3.2.2), bf16, head size 64.
 //
-// One CTA = 64 consecutive tokens of one (batch entry, head), 8 warps.  As in the tiled forward
+// One CTA = 64 consecutive tokens of one (batch entry, head), 8 or 4 warps (see BwdTileCfg).  As in the tiled forward
 // the nodes a token attends at one (side, level) are one contiguous range, so per chunk the CTA
 // stages the union range of K and V rows once.  The token's self loop is folded into the
 // level-0 left chunk: node i follows its left neighbours directly, and the relation ids
 // self = 0, left(0, o) = 1 + o are consecutive, so the self loop is simply offset 0 of a range
 // that ends at the token itself.
 //
-//   phase 1 (two warps share 16 query rows and take the key blocks in turn):  S = Q K^T + skewed Q R^T,  P = exp(S - lse),
+//   phase 1 (16 query rows per warp, or per pair of warps that split every key block):  S = Q K^T + skewed Q R^T,  P = exp(S - lse),
 //            dP = dO V^T,  dS = P (dP - dO.O);  dQ += dS K + skew(dS) R;
 //            P, dS and the skewed dS (indexed by relation offset) go to shared memory as bf16
 //   phase 2 (a warp owns 16 staged key rows):  dK_part = dS^T Q,  dV_part = P^T dO for the

@@ -1,6 +1,6 @@
 // Building blocks of the tcgen05 (5th-generation tensor core) kernels: shared-memory matrix
-// descriptors, the instruction descriptor, MMA issue / commit, mbarrier waits with an iteration
-// limit, tensor-memory allocation and loads.
+// descriptors, the instruction descriptor, MMA issue / commit, time-bounded mbarrier waits, TMA
+// tile loads, tensor-memory allocation and loads.
 //
 // Operand tiles live in shared memory as rows of 128 bytes (64 bf16) whose eight 16-byte chunks
 // are XOR-swizzled with the row index modulo 8 -- the layout tile_off() of mma_tools.cuh writes,
