@@ -135,24 +135,24 @@ class MaskedGraph:
         self.n_edges = int(self.col.shape[0])
 
 
-def attn_fwd_varlen(g, q, k, v, r, scale, lengths):
-    """Forward with one length per batch entry."""
+def attn_fwd_varlen(g, q, k, v, r, scale, lengths, p_drop=0.0, seed=0):
+    """Forward with one length per batch entry (and, optionally, attention dropout)."""
     q = _f64(q)
     out = np.zeros_like(q)
     lse = np.zeros(q.shape[:3])
     for b, length in enumerate(lengths):
-        o, l = attn_fwd(MaskedGraph(g, int(length)), q, k, v, r, scale, b0=b, b1=b + 1)
+        o, l = attn_fwd(MaskedGraph(g, int(length)), q, k, v, r, scale, b0=b, b1=b + 1, p_drop=p_drop, seed=seed)
         out[b], lse[b] = o[b], l[b]
     return out, lse
 
 
-def attn_bwd_varlen(g, q, k, v, r, scale, d_out, lengths, out=None):
-    """Backward with one length per batch entry; dr sums over the batch."""
+def attn_bwd_varlen(g, q, k, v, r, scale, d_out, lengths, out=None, p_drop=0.0, seed=0):
+    """Backward with one length per batch entry (and, optionally, attention dropout); dr sums over the batch."""
     q = _f64(q)
     dq, dk, dv = np.zeros_like(q), np.zeros_like(q), np.zeros_like(q)
     dr = np.zeros_like(_f64(r))
     for b, length in enumerate(lengths):
-        a = attn_bwd(MaskedGraph(g, int(length)), q, k, v, r, scale, d_out, b0=b, b1=b + 1, out=out)
+        a = attn_bwd(MaskedGraph(g, int(length)), q, k, v, r, scale, d_out, b0=b, b1=b + 1, out=out, p_drop=p_drop, seed=seed)
         dq[b], dk[b], dv[b] = a[0][b], a[1][b], a[2][b]
         dr += a[3]
     return dq, dk, dv, dr
