@@ -56,7 +56,9 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-template <bool kDrop>  // attention dropout compiled in or out: the plain kernel carries none of it
+// kDrop: attention dropout compiled in or out (the plain kernel carries none of it).  NG: 16-key groups per
+// step of the key loop (2 = 32 keys; 1 = 16 keys, which skips more of the masked columns when k is small).
+template <bool kDrop, int NG>
 __global__ void __launch_bounds__(128)
 fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
                 const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
@@ -224,14 +226,14 @@ fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
         const int2 ba = bc[r0 + g], bb = bc[r0 + g + 8];
         const int lo_r[2] = {ba.x, bb.x}, hi_r[2] = {ba.y, bb.y};
         const int kstart = (wr.x - base) & ~15, kend = wr.y - base;
-        for (int kb = kstart; kb <= kend; kb += 32) {
-            float s[4][4];
+        for (int kb = kstart; kb <= kend; kb += 16 * NG) {
+            float s[2 * NG][4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+            for (int j = 0; j < 2 * NG; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks) {
 #pragma unroll
-                for (int np = 0; np < 2; ++np) {
+                for (int np = 0; np < NG; ++np) {
                     uint32_t bf[4];
                     load_b_rows(k_u, kb + np * 16, ks, lane, bf);
                     mma_bf16(s[np * 2], qa[ks], bf[0], bf[1]);
@@ -241,7 +243,7 @@ fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
             // relative-position term, mask, running max
             float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < 2 * NG; ++j) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const int hh = e >> 1;
@@ -271,9 +273,9 @@ fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
                 o[nt][0] *= corr[0]; o[nt][1] *= corr[0];
                 o[nt][2] *= corr[1]; o[nt][3] *= corr[1];
             }
-            uint32_t pa[2][4];
+            uint32_t pa[NG][4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
+            for (int j = 0; j < 2 * NG; ++j) {
                 float p0 = ex2(s[j][0] - m_run[0]), p1 = ex2(s[j][1] - m_run[0]);
                 float p2 = ex2(s[j][2] - m_run[1]), p3 = ex2(s[j][3] - m_run[1]);
                 l_run[0] += p0 + p1;
@@ -288,7 +290,7 @@ fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
                 pa[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
             }
 #pragma unroll
-            for (int kk = 0; kk < 2; ++kk) {
+            for (int kk = 0; kk < NG; ++kk) {
 #pragma unroll
                 for (int np = 0; np < 4; ++np) {
                     uint32_t bf[4];
@@ -338,7 +340,9 @@ bpt_status launch_fwd_tile(const AttnProblem& p) {
     context_levels(p.tree, &n_left, &n_right);
     const FwdTileCfg cfg = make_fwd_tile_cfg(p.tree, n_left + n_right);
     const size_t smem = cfg.bytes;
-    auto kernel = p.drop.thr ? fwd_tile_kernel<true> : fwd_tile_kernel<false>;
+    const bool narrow = p.tree.k <= 8;  // measured: 16-key steps win a few percent for k <= 8 and lose at k = 16
+    auto kernel = p.drop.thr ? (narrow ? fwd_tile_kernel<true, 1> : fwd_tile_kernel<true, 2>)
+                             : (narrow ? fwd_tile_kernel<false, 1> : fwd_tile_kernel<false, 2>);
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
         return BPT_ERR_CUDA;
     if (smem > 200 * 1024 || p.H > 65535 || p.B > 65535) return BPT_ERR_UNSUPPORTED;
