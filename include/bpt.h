@@ -15,7 +15,8 @@
  * Ownership: the caller owns every buffer.  Unless a comment says "host", every
  * pointer is a DEVICE pointer valid on the current device.  Calls enqueue work on
  * `cuda_stream` (a cudaStream_t passed as void*, NULL = legacy default stream) and
- * return without synchronising.  Nothing is allocated or kept between calls.
+ * return without synchronising.  Nothing is allocated or kept between calls, so the attention calls
+ * (bpt_attn_fwd / bpt_attn_bwd and their _varlen, _ex, _rows forms) can be captured in a CUDA graph.
  * Argument errors are detected on the host before anything is launched.
  */
 #ifndef BPT_H
