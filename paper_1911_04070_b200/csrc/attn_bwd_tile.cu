@@ -17,6 +17,8 @@
 // Nothing is accumulated across CTAs here: bwd_gather_kernel sums, for every source node, the
 // partial rows of the tiles whose range covers it, in tile order (no atomics, fixed order), and
 // drel_sum kernels do the same for the relation table.
+#include <cstdlib>
+
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
 #include "row_map.cuh"
@@ -603,7 +605,16 @@ struct TileWorkspace {
     size_t bytes;
 };
 
-constexpr size_t kPassBytes = (size_t)3 << 30;  // partial rows kept per pass
+// Partial rows kept per pass over the (batch entry, head) pairs: 10 GiB, or BPT_BWD_PASS_MB from the
+// environment (read once; smaller values trade workspace for more passes).
+size_t pass_bytes() {
+    static const size_t v = [] {
+        const char* e = getenv("BPT_BWD_PASS_MB");
+        const long mb = e ? atol(e) : 0;
+        return mb > 0 ? (size_t)mb << 20 : (size_t)10 << 30;
+    }();
+    return v;
+}
 
 ChunkPlan make_plan(const TreeParams& t) {
     ChunkPlan p{};
@@ -625,7 +636,7 @@ TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, int B, int 
     const size_t per_pair = ((size_t)tiles * ((size_t)plan.slab_row0[chunks] * 128 + (size_t)chunks * plan.rel_store * 64) +
                              bwd_span_slab_floats(t, 1) + bwd_span_ext_floats(t, 1)) * sizeof(float);
     TileWorkspace w;
-    size_t pairs = kPassBytes / per_pair;
+    size_t pairs = pass_bytes() / per_pair;
     if (pairs < 1) pairs = 1;
     if (pairs > (size_t)B * H) pairs = (size_t)B * H;
     w.pairs_per_pass = (int)pairs;
