@@ -68,7 +68,7 @@ def all_configs():
 
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples during the timed region."""
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -82,12 +82,13 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Samples taken between the two host times (time.time()) when given and any fall inside, else all."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -96,24 +97,31 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        import datetime
+        rows = []
         try:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
-                if len(f) < 9:
+                if len(f) < 10:
                     continue
                 try:
-                    sm.append(float(f[1])); mx.append(float(f[2]))
+                    ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(f[2]), float(f[3]), f[6:10]))
                 except ValueError:
                     continue
-                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
             os.unlink(self.path)
         except OSError:
             pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        inside = [r for r in rows if t_begin is not None and t_begin - 0.02 <= r[0] <= t_end + 0.02]
+        use = inside or rows
+        if use:
+            reasons = set()
+            for r in use:
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            out.update(sm_mhz=statistics.median(r[1] for r in use), sm_max_mhz=max(r[2] for r in use), reasons=sorted(reasons),
+                       samples=len(use), window="timed region" if inside else "warm-up and timed region")
         return out
 
 
@@ -236,14 +244,18 @@ def run_ours(args, cfg_name, cfg):
         dist.all_reduce(v, op=dist.ReduceOp.MAX)
         return float(v.item())
 
+    sampler = ClockSampler(local_rank)   # started before the warm-up: nvidia-smi takes a moment to deliver samples
+    if rank == 0:
+        sampler.start()
     for _ in range(args.warmup):
+        step()
+    barrier()
+    t_load = time.time()
+    while time.time() - t_load < 0.3:    # keep the GPU under the same load until the sampler is up (untimed)
         step()
     barrier()
 
     # ---- timed region: K steps, device-resident inputs ---------------------------------
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
     cap = min(args.steps * 16 + 8, 4000)
     # L2 (126 MB): a workload whose tensors exceed it evicts itself between steps; a smaller one gets a
     # 256 MB write between the timed steps, which are then timed one by one
@@ -252,6 +264,7 @@ def run_ours(args, cfg_name, cfg):
     scrub = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev) if flush else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    t_begin = time.time()
     if not flush:
         binding.bpt_trace_begin(cap)
         e0.record()
@@ -273,8 +286,9 @@ def run_ours(args, cfg_name, cfg):
             ms_sum += e0.elapsed_time(e1)
             marks += binding.bpt_trace_end(16)
         barrier()
+    t_end = time.time()
     ms_total = max_over_ranks(ms_sum)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     ms_step = ms_total / args.steps
     value = world * B * E / (ms_step * 1e-3)
 
