@@ -102,6 +102,10 @@ bpt_status bpt_build_graph(const bpt_graph_dims* dims, int32_t* row_ptr, int32_t
 /*
  * Bytes of device workspace bpt_attn_fwd (backward == 0) or bpt_attn_bwd
  * (backward != 0) needs for this problem; 0 on invalid arguments.  Host only.
+ * The tiled backward keeps partial gradient rows of as many (batch entry, head) pairs as fit
+ * 10 GiB and works through larger problems in passes; BPT_BWD_PASS_MB in the environment (read
+ * once per process) sets another cap in MiB, trading workspace for passes.  The same sizes serve
+ * the _varlen and _ex forms.
  */
 size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype, int backward);
 
