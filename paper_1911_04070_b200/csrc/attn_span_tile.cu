@@ -257,32 +257,36 @@ fwd_span_merge_kernel(TreeParams t, const float* __restrict__ ext_part, __nv_bfl
     const int T0 = mi << (j - kInnerLevels), nT = 1 << (j - kInnerLevels);
     const float* base = ext_part + (((size_t)pair * tiles + T0) * n_ext + e) * kExtStride;
     const size_t stride = (size_t)n_ext * kExtStride;
+    // lane t takes tiles t, t + 32, ...; the lanes' sums are then added in a fixed butterfly order
     float mx = -INFINITY;
     for (int x = lane; x < nT; x += 32) mx = fmaxf(mx, base[(size_t)x * stride]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (mx == -INFINITY) mx = 0.f;  // a span without real tokens: every partial is empty (2^-inf = 0 below)
-    // tiles sixteen at a time: all loads of a batch are issued before any of them is used; summed in tile order
-    float l = 0.f, a0 = 0.f, a1 = 0.f;
-    for (int x0 = 0; x0 < nT; x0 += 16) {
-        float mm[16], ll[16];
-        float2 aa[16];
+    float l = 0.f, acc[64];
 #pragma unroll
-        for (int u = 0; u < 16; ++u) {
-            const bool in = x0 + u < nT;
-            const float* p = base + (size_t)(in ? x0 + u : 0) * stride;
-            mm[u] = in ? p[0] : -INFINITY;
-            ll[u] = p[1];
-            aa[u] = *reinterpret_cast<const float2*>(p + 2 + lane * 2);
-        }
+    for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+    for (int x = lane; x < nT; x += 32) {
+        const float* p = base + (size_t)x * stride;
+        const float f = fast_exp2(p[0] - mx);
+        l = fmaf(p[1], f, l);
 #pragma unroll
-        for (int u = 0; u < 16; ++u) {
-            const float f = fast_exp2(mm[u] - mx);  // 0 for the slots past the last tile
-            l = fmaf(ll[u], f, l);
-            a0 = fmaf(aa[u].x, f, a0);
-            a1 = fmaf(aa[u].y, f, a1);
+        for (int c = 0; c < 32; ++c) {
+            const float2 a = *reinterpret_cast<const float2*>(p + 2 + 2 * c);
+            acc[2 * c] = fmaf(a.x, f, acc[2 * c]);
+            acc[2 * c + 1] = fmaf(a.y, f, acc[2 * c + 1]);
         }
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        l += __shfl_xor_sync(0xffffffffu, l, o);
+#pragma unroll
+        for (int c = 0; c < 64; ++c) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+    }
+    float a0 = 0.f, a1 = 0.f;  // this lane's two channels (static register indices only)
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+        if (c == lane) { a0 = acc[2 * c]; a1 = acc[2 * c + 1]; }
     const float inv = l > 0.f ? 1.f / l : 0.f;  // l = 0: a span without real tokens
     const size_t rs = (size_t)H * 64;
     *reinterpret_cast<uint32_t*>(out + ((size_t)b * (2 * t.n - 1) + node) * rs + (size_t)h * 64 + lane * 2) = pack_bf16(a0 * inv, a1 * inv);
@@ -541,15 +545,29 @@ bwd_span_merge_kernel(TreeParams t, const float* __restrict__ ext_dq, __nv_bfloa
     const int node = 2 * t.n - 2 - (int)(wid % n_outer);
     const int j = node_level(t.n, node), mi = node - node_id(t.n, j, 0), e = j - kInnerLevels - 1;
     const int T0 = mi << (j - kInnerLevels), nT = 1 << (j - kInnerLevels);
-    const float* base = ext_dq + (((size_t)pl * tiles + T0) * n_ext + e) * 64 + lane * 2;
+    const float* base = ext_dq + (((size_t)pl * tiles + T0) * n_ext + e) * 64;
     const size_t stride = (size_t)n_ext * 64;
-    float a0 = 0.f, a1 = 0.f;
-#pragma unroll 16
-    for (int x = 0; x < nT; ++x) {
-        const float2 a = *reinterpret_cast<const float2*>(base + (size_t)x * stride);
-        a0 += a.x;
-        a1 += a.y;
+    // lane t takes tiles t, t + 32, ...; the lanes' sums are then added in a fixed butterfly order
+    float acc[64];
+#pragma unroll
+    for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+    for (int x = lane; x < nT; x += 32) {
+        const float4* p = reinterpret_cast<const float4*>(base + (size_t)x * stride);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+            const float4 a = p[c];
+            acc[4 * c] += a.x; acc[4 * c + 1] += a.y; acc[4 * c + 2] += a.z; acc[4 * c + 3] += a.w;
+        }
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+        for (int c = 0; c < 64; ++c) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
+    }
+    float a0 = 0.f, a1 = 0.f;  // this lane's two channels (static register indices only)
+#pragma unroll
+    for (int c = 0; c < 32; ++c)
+        if (c == lane) { a0 = acc[2 * c]; a1 = acc[2 * c + 1]; }
     const size_t rs = (size_t)H * 64;
     *reinterpret_cast<uint32_t*>(dq + ((size_t)b * (2 * t.n - 1) + node) * rs + (size_t)h * 64 + lane * 2) = pack_bf16(a0 * scale, a1 * scale);
 }
