@@ -76,16 +76,22 @@ constexpr BwdTileCfg layout_of(int kv_rows, int rel_rows, int qr_stride) {
     c.bnd_off = c.row_off + 2 * kTileTokens * 4;
     return c;
 }
+constexpr size_t kTwoCtaBytes = 112 * 1024;  // shared memory per CTA up to which two CTAs fit an SM
 // the sizes of k = 64: the eight-warp kernel has this layout as compile-time constants
 constexpr BwdTileCfg kWidestCfg = layout_of(kMaxKvRows, kMaxRelRows, kMaxRelRows - 4);
 
 BwdTileCfg make_bwd_tile_cfg(const TreeParams& t, int chunks, bool widest) {
     BwdTileCfg c = kWidestCfg;
+    const size_t tail = (size_t)chunks * (kTileTokens * 8 + 8);
     if (!widest) {
+        // widest buffers that still let two CTAs share an SM; ranges wider than that go in sub-blocks
         const int rel_rows = min(kMaxRelRows, (t.k + 2 + 15) & ~15);
-        c = layout_of(min(kMaxKvRows, (t.kc + 143) & ~15), rel_rows, rel_rows - 4 >= t.k + 2 ? rel_rows - 4 : rel_rows + 4);
+        const int qr_stride = rel_rows - 4 >= t.k + 2 ? rel_rows - 4 : rel_rows + 4;
+        int kv_rows = min(kMaxKvRows, (t.kc + 97) & ~15);  // 15 (alignment) + 64 + k + 3 columns at most, rounded up to 16
+        while (kv_rows > 64 && layout_of(kv_rows, rel_rows, qr_stride).bnd_off + tail > kTwoCtaBytes) kv_rows -= 16;
+        c = layout_of(kv_rows, rel_rows, qr_stride);
     }
-    c.bytes = (size_t)c.bnd_off + (size_t)chunks * (kTileTokens * 8 + 8);
+    c.bytes = (size_t)c.bnd_off + tail;
     return c;
 }
 
@@ -100,7 +106,7 @@ __device__ __forceinline__ void pair_barrier(int rg) {
 }
 
 struct ChunkGeom {
-    int side, level, n_l, id_base, rel_base, n_rel_c, base, kend, nr;
+    int side, level, n_l, id_base, rel_base, n_rel_c, base, kend;
 };
 
 __device__ __forceinline__ ChunkGeom chunk_geom(const TreeParams& t, int n_left, int c, int2 cr) {
@@ -113,7 +119,6 @@ __device__ __forceinline__ ChunkGeom chunk_geom(const TreeParams& t, int n_left,
     gm.n_rel_c = c == 0 ? t.k + 2 : t.k + 1;  // chunk 0 also holds r^self
     gm.base = cr.x & ~15;
     gm.kend = cr.y - gm.base;
-    gm.nr = (gm.kend + 1 + 31 + 15) & ~15;  // capped by the caller's buffer
     return gm;
 }
 
@@ -221,21 +226,26 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
     float* slab_cta = slabs + ((size_t)blockIdx.y * tiles + tile) * plan.slab_row0[chunks] * 128;
     float* drel_cta = drel_part + ((size_t)blockIdx.y * tiles + tile) * chunks * plan.rel_store * 64;
 
-    // K / V rows of the chunk's node range and its relation rows -> shared memory (async)
-    auto stage = [&](int c) {
+    // A chunk whose node range is wider than the K / V buffers is worked through in sub-blocks of
+    // cfg.kv_rows columns; (c, s0) = chunk and first column of the sub-block.  Its length:
+    auto sub_len = [&](const ChunkGeom& gm, int s0) { return min(cfg.kv_rows, (gm.kend + 1 - s0 + 15) & ~15); };
+    // K / V rows of the sub-block and, with its first sub-block, the chunk's relation rows -> shared memory (async)
+    auto stage = [&](int c, int s0) {
         const ChunkGeom gm = chunk_geom(t, n_left, c, crange[c]);
-        const int nr = min(cfg.kv_rows, gm.nr);
+        const int nr = sub_len(gm, s0);
         for (int idx = tid; idx < nr * 8; idx += kBwdThreads) {
             const int row = idx >> 3, ch = idx & 7;
-            const int node = min(gm.base + row, gm.n_l - 1);
+            const int node = min(gm.base + s0 + row, gm.n_l - 1);  // rows past the range repeat a real row: finite values
             const size_t src = boff + (size_t)(gm.id_base + node) * rs + ch * 8;
             cp_async16(k_u + tile_off(row, ch), k + src);
             cp_async16(v_u + tile_off(row, ch), v + src);
         }
-        for (int idx = tid; idx < cfg.rel_rows * 8; idx += kBwdThreads) {
-            const int row = idx >> 3, ch = idx & 7;
-            if (row < gm.n_rel_c) cp_async16(r_u + tile_off(row, ch), r + (size_t)(gm.rel_base + row) * 64 + ch * 8);
-            else *reinterpret_cast<uint4*>(r_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
+        if (s0 == 0) {
+            for (int idx = tid; idx < cfg.rel_rows * 8; idx += kBwdThreads) {
+                const int row = idx >> 3, ch = idx & 7;
+                if (row < gm.n_rel_c) cp_async16(r_u + tile_off(row, ch), r + (size_t)(gm.rel_base + row) * 64 + ch * 8);
+                else *reinterpret_cast<uint4*>(r_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
+            }
         }
     };
 
@@ -245,24 +255,28 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
         if (tid < kTileTokens) mask_row_bounds(t, t0, tid, n_left, n_right, bnd, len);
     }
     __syncthreads();  // delta and crange are visible; the out tile in the K buffer is consumed
-    stage(0);         // chunk 0 (left level 0 with the self loop) is never empty
+    stage(0, 0);      // chunk 0 (left level 0 with the self loop) is never empty
     cp_async_commit();
 
-    int c = 0;
+    int c = 0, s0 = 0;
     while (c < chunks) {
-        for (int idx = tid; idx < kTileTokens * (kSkewStride / 16); idx += kBwdThreads)
-            *reinterpret_cast<uint4*>(sk_s + idx * 16) = make_uint4(0, 0, 0, 0);
-        cp_async_wait<0>();
-        __syncthreads();
         const int2 cr = crange[c];
         const ChunkGeom gm = chunk_geom(t, n_left, c, cr);
-        const int side = gm.side, base = gm.base, kend = gm.kend, n_rel_c = gm.n_rel_c;
+        const int side = gm.side, n_rel_c = gm.n_rel_c;
+        const int sb_len = sub_len(gm, s0);                      // columns of this sub-block (a multiple of 16)
+        const bool first = s0 == 0, last = s0 + sb_len > gm.kend;  // first / last sub-block of the chunk
+        const int base = gm.base + s0;                           // node index of the sub-block's column 0
+        if (first)
+            for (int idx = tid; idx < kTileTokens * (kSkewStride / 16); idx += kBwdThreads)
+                *reinterpret_cast<uint4*>(sk_s + idx * 16) = make_uint4(0, 0, 0, 0);
+        cp_async_wait<0>();
+        __syncthreads();
 
         // ================= phase 1: 16 query rows per pair of warps, key blocks alternate =================
         const int2* bc = bnd + c * kTileTokens;
         const int2 wr = rows_union(bc, r0, 16, lane);
         const bool w_any = wr.x <= wr.y;
-        if (w_any) {  // Q R^T for the chunk's relation rows -> the row group's scratch
+        if (w_any && first) {  // Q R^T for the chunk's relation rows -> the row group's scratch (kept for all sub-blocks)
 #pragma unroll
             for (int np = 0; np < kMaxRelRows / 16; ++np) {
                 if (np * 16 < n_rel_c && (!kPair || (np & 1) == half)) {
@@ -372,16 +386,16 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
                 }
             }
         };
-        for (int kb0 = 0; kb0 <= kend; kb0 += 32) {
+        for (int kb0 = 0; kb0 < sb_len; kb0 += 32) {
             if constexpr (kPair) {
-                keys(kb0 + half * 16);
+                if (kb0 + half * 16 < sb_len) keys(kb0 + half * 16);
             } else {
                 keys(kb0);
-                keys(kb0 + 16);
+                if (kb0 + 16 < sb_len) keys(kb0 + 16);
             }
         }
         if constexpr (kPair) pair_barrier(rg); else __syncwarp();  // the group's rows of the skew tile are complete
-        if (w_any) {       // dQ += skew(dS) R_chunk, the k-steps shared out between the two warps
+        if (w_any && last) {  // dQ += skew(dS) R_chunk once the chunk's skew tile is complete, the k-steps shared out between the two warps
 #pragma unroll
             for (int kk = 0; kk < kMaxRelRows / 16; ++kk) {
                 if (kk * 16 < n_rel_c && (!kPair || (kk & 1) == half)) {
@@ -399,19 +413,23 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
         }
         __syncthreads();  // P, dS and the skew tile are complete; K, V and R tiles are free
 
-        // next chunk that this tile reaches: its K / V / R rows arrive while phase 2 runs
-        int cn = c + 1;
-        while (cn < chunks && crange[cn].x > crange[cn].y) {  // a level no token of the tile reaches: zero d_rel partial
-            float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)cn * plan.rel_store * 64);
-            for (int idx = tid; idx < plan.rel_store * 16; idx += kBwdThreads) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-            ++cn;
+        // next sub-block, or the next chunk that this tile reaches: its rows arrive while phase 2 runs
+        int cn = c, sn = s0 + sb_len;
+        if (last) {
+            cn = c + 1;
+            sn = 0;
+            while (cn < chunks && crange[cn].x > crange[cn].y) {  // a level no token of the tile reaches: zero d_rel partial
+                float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)cn * plan.rel_store * 64);
+                for (int idx = tid; idx < plan.rel_store * 16; idx += kBwdThreads) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+                ++cn;
+            }
         }
-        if (cn < chunks) stage(cn);
+        if (cn < chunks) stage(cn, sn);
         cp_async_commit();
 
         // ================= phase 2: key tiles (dk, dv partial rows) and offset tiles (d_rel partial) =================
         // jobs: (key tile | offset tile) x (channels 0..31 | 32..63); key-tile jobs are twice as heavy, so they go first
-        const int n_jt = (kend >> 4) + 1, n_ot = plan.rel_rows >> 4;
+        const int n_jt = sb_len >> 4, n_ot = last ? plan.rel_rows >> 4 : 0;  // the d_rel tiles once per chunk
         for (int job = w; job < 2 * (n_jt + n_ot); job += kBwdThreads / 32) {
             const int hc = job & 1, tile16 = job >> 1;  // channel half, tile
             if (tile16 < n_jt) {
@@ -481,6 +499,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
         }
         __syncthreads();  // P, dS and skew tiles are free again
         c = cn;
+        s0 = sn;
     }
 
     // ---- epilogue: the two warps' dq parts are added (second warp's part through shared memory), ----
@@ -671,7 +690,7 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
     const int chunks = plan.n_left + plan.n_right, tiles = t.n / kTileTokens, N = 2 * t.n - 1;
     const TileWorkspace ws = carve_tile(t, plan, p.B, p.H, p.workspace);
     BwdTileCfg cfg = make_bwd_tile_cfg(t, chunks, false);
-    const bool four = cfg.bytes <= 112 * 1024;  // two CTAs fit an SM: four warps each, independent barriers
+    const bool four = cfg.bytes <= kTwoCtaBytes;  // two CTAs fit an SM: four warps each, independent barriers
     if (!four) cfg = make_bwd_tile_cfg(t, chunks, true);
     const size_t smem = cfg.bytes;
     if (smem > 227 * 1024) return BPT_ERR_UNSUPPORTED;
