@@ -1,14 +1,15 @@
 // Tiled backward for the token rows (arXiv 1911.04070: gradient of the Sec. 3.4 equation over
 // the contextual edges of Sec. 3.2.2), bf16, head size 64.
 //
-// One CTA = 64 consecutive tokens of one (batch entry, head), 8 or 4 warps (see BwdTileCfg).  As in the tiled forward
+// One CTA = 64 consecutive tokens of one (batch entry, head), 4 warps (16 query rows each); the buffers
+// are sized so that two CTAs share an SM (see BwdTileCfg).  As in the tiled forward
 // the nodes a token attends at one (side, level) are one contiguous range, so per chunk the CTA
 // stages the union range of K and V rows once.  The token's self loop is folded into the
 // level-0 left chunk: node i follows its left neighbours directly, and the relation ids
 // self = 0, left(0, o) = 1 + o are consecutive, so the self loop is simply offset 0 of a range
 // that ends at the token itself.
 //
-//   phase 1 (16 query rows per warp, or per pair of warps that split every key block):  S = Q K^T + skewed Q R^T,  P = exp(S - lse),
+//   phase 1 (16 query rows per warp):  S = Q K^T + skewed Q R^T,  P = exp(S - lse),
 //            dP = dO V^T,  dS = P (dP - dO.O);  dQ += dS K + skew(dS) R;
 //            P, dS and the skewed dS (indexed by relation offset) go to shared memory as bf16
 //   phase 2 (a warp owns 16 staged key rows):  dK_part = dS^T Q,  dV_part = P^T dO for the
@@ -45,8 +46,9 @@ struct ChunkPlan {
     int rel_store;                  // rows kept per chunk in the d_rel partials: k + 2, the most a chunk uses
 };
 
-// Shared-memory layout; the buffer sizes follow k.  Where two CTAs fit an SM the kernel runs with four
-// warps per CTA (one per group of 16 query rows), otherwise with eight (two per group).
+// Shared-memory layout.  The buffer sizes follow k and are capped so that two CTAs fit an SM (two
+// independent CTAs of four warps measured 10 to 30 % faster than one CTA of eight warps that share
+// barriers); a chunk whose node range is wider than the K / V buffers is worked through in sub-blocks.
 struct BwdTileCfg {
     int kv_rows;      // staged K / V rows (multiple of 16)
     int rel_rows;     // staged relation rows (multiple of 16)
@@ -77,32 +79,16 @@ constexpr BwdTileCfg layout_of(int kv_rows, int rel_rows, int qr_stride) {
     return c;
 }
 constexpr size_t kTwoCtaBytes = 112 * 1024;  // shared memory per CTA up to which two CTAs fit an SM
-// the sizes of k = 64: the eight-warp kernel has this layout as compile-time constants
-constexpr BwdTileCfg kWidestCfg = layout_of(kMaxKvRows, kMaxRelRows, kMaxRelRows - 4);
 
-BwdTileCfg make_bwd_tile_cfg(const TreeParams& t, int chunks, bool widest) {
-    BwdTileCfg c = kWidestCfg;
+BwdTileCfg make_bwd_tile_cfg(const TreeParams& t, int chunks) {
     const size_t tail = (size_t)chunks * (kTileTokens * 8 + 8);
-    if (!widest) {
-        // widest buffers that still let two CTAs share an SM; ranges wider than that go in sub-blocks
-        const int rel_rows = min(kMaxRelRows, (t.k + 2 + 15) & ~15);
-        const int qr_stride = rel_rows - 4 >= t.k + 2 ? rel_rows - 4 : rel_rows + 4;
-        int kv_rows = min(kMaxKvRows, (t.kc + 97) & ~15);  // 15 (alignment) + 64 + k + 3 columns at most, rounded up to 16
-        while (kv_rows > 64 && layout_of(kv_rows, rel_rows, qr_stride).bnd_off + tail > kTwoCtaBytes) kv_rows -= 16;
-        c = layout_of(kv_rows, rel_rows, qr_stride);
-    }
+    const int rel_rows = min(kMaxRelRows, (t.k + 2 + 15) & ~15);
+    const int qr_stride = rel_rows - 4 >= t.k + 2 ? rel_rows - 4 : rel_rows + 4;
+    int kv_rows = min(kMaxKvRows, (t.kc + 97) & ~15);  // 15 (alignment) + 64 + k + 3 columns at most, rounded up to 16
+    while (kv_rows > 64 && layout_of(kv_rows, rel_rows, qr_stride).bnd_off + tail > kTwoCtaBytes) kv_rows -= 16;
+    BwdTileCfg c = layout_of(kv_rows, rel_rows, qr_stride);
     c.bytes = (size_t)c.bnd_off + tail;
     return c;
-}
-
-// barrier of the two warps that share a group of query rows (ids 1..4; id 0 is __syncthreads)
-__device__ __forceinline__ void pair_barrier(int rg) {
-    switch (rg) {
-        case 0: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
-        case 1: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
-        case 2: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
-        default: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
-    }
 }
 
 struct ChunkGeom {
@@ -122,9 +108,10 @@ __device__ __forceinline__ ChunkGeom chunk_geom(const TreeParams& t, int n_left,
     return gm;
 }
 
-template <int NW>  // warps per CTA: 8 (two per group of 16 query rows) or 4 (one per group)
-__global__ void __launch_bounds__(NW * 32)
-bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
+constexpr int kBwdThreads = 128;  // 4 warps, one per group of 16 query rows
+
+__global__ void __launch_bounds__(kBwdThreads)
+bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
                 const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                 const __nv_bfloat16* __restrict__ v, const __nv_bfloat16* __restrict__ r,
                 const __nv_bfloat16* __restrict__ out, const float* __restrict__ lse,
@@ -132,7 +119,6 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
                 int2* __restrict__ tile_range, float* __restrict__ slabs, float* __restrict__ drel_part,
                 int H, int pair0, float scale, const int32_t* __restrict__ lengths, DropoutParams drop) {
     extern __shared__ __align__(128) unsigned char smem[];
-    const BwdTileCfg cfg = NW == 8 ? kWidestCfg : cfg_arg;  // eight warps: the widest layout, all constants
     unsigned char* q_s = smem;
     unsigned char* g_s = smem + cfg.g_off;   // d_out tile
     unsigned char* k_s = smem + cfg.k_off;
@@ -149,10 +135,8 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
     int2* crange = bnd + chunks * kTileTokens;
 
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    constexpr int kBwdThreads = NW * 32;
-    constexpr bool kPair = NW == 8;
     const int kQrStride = cfg.qr_stride, kPStride = cfg.p_stride, kSkewStride = cfg.skew_stride;
-    const int rg = w & 3, half = kPair ? w >> 2 : 0;  // row group (16 query rows) and, with eight warps, which of its two warps
+    const int rg = w;  // row group: this warp's 16 query rows
     const int g = lane >> 2, c2 = (lane & 3) * 2;
     const int tile = blockIdx.x, tiles = gridDim.x, t0 = tile * kTileTokens;
     const int pair = pair0 + blockIdx.y, b = pair / H, h = pair % H;
@@ -279,7 +263,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
         if (w_any && first) {  // Q R^T for the chunk's relation rows -> the row group's scratch (kept for all sub-blocks)
 #pragma unroll
             for (int np = 0; np < kMaxRelRows / 16; ++np) {
-                if (np * 16 < n_rel_c && (!kPair || (np & 1) == half)) {
+                if (np * 16 < n_rel_c) {
                     float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
@@ -299,17 +283,15 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
                 }
             }
         }
-        if constexpr (kPair) pair_barrier(rg); else __syncwarp();
+        __syncwarp();
 
         const int2 ba = bc[r0 + g], bb = bc[r0 + g + 8];
         const int lo_r[2] = {ba.x, bb.x}, hi_r[2] = {ba.y, bb.y};
         const float lse_r[2] = {lse_s[r0 + g], lse_s[r0 + g + 8]};
         const float del_r[2] = {delta_s[r0 + g], delta_s[r0 + g + 8]};
         const int w_lo = w_any ? wr.x - base : 1 << 30, w_hi = w_any ? wr.y - base : -1;
-        // 16 * NG keys of a block: S, dP, the element-wise part, P / dS / skew to shared memory, dQ += dS K.
-        // With eight warps the two warps of a row group take 16 keys each of every 32-key block (balanced
-        // whatever the block count); with four warps a warp takes both halves in turn (16-key granularity
-        // skips more of the masked columns at small k than whole blocks would: measured 0.77 against 0.83 ms at k = 8).
+        // 16 keys at a time: S, dP, the element-wise part, P / dS / skew to shared memory, dQ += dS K.  (16-key
+        // granularity skips more of the masked columns than 32 would: measured 0.77 against 0.83 ms at k = 8.)
         constexpr int NG = 1;
         auto keys = [&](int kb) {
             unsigned char* p_row0 = p_s + (r0 + g) * kPStride + (kb + c2) * 2;
@@ -387,18 +369,14 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
             }
         };
         for (int kb0 = 0; kb0 < sb_len; kb0 += 32) {
-            if constexpr (kPair) {
-                if (kb0 + half * 16 < sb_len) keys(kb0 + half * 16);
-            } else {
-                keys(kb0);
-                if (kb0 + 16 < sb_len) keys(kb0 + 16);
-            }
+            keys(kb0);
+            if (kb0 + 16 < sb_len) keys(kb0 + 16);
         }
-        if constexpr (kPair) pair_barrier(rg); else __syncwarp();  // the group's rows of the skew tile are complete
+        __syncwarp();  // this warp's rows of the skew tile are complete
         if (w_any && last) {  // dQ += skew(dS) R_chunk once the chunk's skew tile is complete, the k-steps shared out between the two warps
 #pragma unroll
             for (int kk = 0; kk < kMaxRelRows / 16; ++kk) {
-                if (kk * 16 < n_rel_c && (!kPair || (kk & 1) == half)) {
+                if (kk * 16 < n_rel_c) {
                     uint32_t a[4];
                     load_a_plain(sk_u, kSkewStride, r0, kk * 16, lane, a);
 #pragma unroll
@@ -502,33 +480,17 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg_arg,
         s0 = sn;
     }
 
-    // ---- epilogue: the two warps' dq parts are added (second warp's part through shared memory), ----
-    // ---- dq = scale * sum, rounded once to bf16, coalesced stores through the Q tile              ----
-    float* red = reinterpret_cast<float*>(p_s) + rg * 16 * 64;  // [16 rows][64] per row group
-    if (kPair && half == 1) {
+    // ---- epilogue: dq = scale * acc, rounded once to bf16, coalesced stores through the Q tile ----
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            *reinterpret_cast<float2*>(red + g * 64 + nt * 8 + c2) = make_float2(acc_q[nt][0], acc_q[nt][1]);
-            *reinterpret_cast<float2*>(red + (g + 8) * 64 + nt * 8 + c2) = make_float2(acc_q[nt][2], acc_q[nt][3]);
-        }
+    for (int nt = 0; nt < 8; ++nt) {
+        *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g, nt) + c2 * 2) = pack_bf16(acc_q[nt][0] * scale, acc_q[nt][1] * scale);
+        *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g + 8, nt) + c2 * 2) = pack_bf16(acc_q[nt][2] * scale, acc_q[nt][3] * scale);
     }
-    __syncthreads();
-    if (half == 0) {
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            const float2 x = kPair ? *reinterpret_cast<const float2*>(red + g * 64 + nt * 8 + c2) : make_float2(0.f, 0.f);
-            const float2 y = kPair ? *reinterpret_cast<const float2*>(red + (g + 8) * 64 + nt * 8 + c2) : make_float2(0.f, 0.f);
-            *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g, nt) + c2 * 2) =
-                pack_bf16((acc_q[nt][0] + x.x) * scale, (acc_q[nt][1] + x.y) * scale);
-            *reinterpret_cast<uint32_t*>(q_s + tile_off(r0 + g + 8, nt) + c2 * 2) =
-                pack_bf16((acc_q[nt][2] + y.x) * scale, (acc_q[nt][3] + y.y) * scale);
-        }
-        __syncwarp();
-        for (int idx = lane; idx < 16 * 8; idx += 32) {
-            const int row = r0 + (idx >> 3), ch = idx & 7;
-            *reinterpret_cast<uint4*>(dq + boff + (size_t)(t0 + row) * rs + ch * 8) =
-                *reinterpret_cast<const uint4*>(q_s + tile_off(row, ch));
-        }
+    __syncwarp();
+    for (int idx = lane; idx < 16 * 8; idx += 32) {
+        const int row = r0 + (idx >> 3), ch = idx & 7;
+        *reinterpret_cast<uint4*>(dq + boff + (size_t)(t0 + row) * rs + ch * 8) =
+            *reinterpret_cast<const uint4*>(q_s + tile_off(row, ch));
     }
 }
 
@@ -689,12 +651,10 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
     const ChunkPlan plan = make_plan(t);
     const int chunks = plan.n_left + plan.n_right, tiles = t.n / kTileTokens, N = 2 * t.n - 1;
     const TileWorkspace ws = carve_tile(t, plan, p.B, p.H, p.workspace);
-    BwdTileCfg cfg = make_bwd_tile_cfg(t, chunks, false);
-    const bool four = cfg.bytes <= kTwoCtaBytes;  // two CTAs fit an SM: four warps each, independent barriers
-    if (!four) cfg = make_bwd_tile_cfg(t, chunks, true);
+    const BwdTileCfg cfg = make_bwd_tile_cfg(t, chunks);
     const size_t smem = cfg.bytes;
     if (smem > 227 * 1024) return BPT_ERR_UNSUPPORTED;
-    auto kernel = four ? bwd_tile_kernel<4> : bwd_tile_kernel<8>;
+    auto kernel = bwd_tile_kernel;
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return BPT_ERR_CUDA;
 
@@ -706,7 +666,7 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
         // span rows: dq of the spans and, per token, the affiliated edges' share of dk / dv
         const bpt_status s = launch_bwd_span(p, pair0, np, ws.ext_dq, ws.aff_slab);
         if (s != BPT_OK) return s;
-        kernel<<<dim3(tiles, np), four ? 128 : 256, smem, p.stream>>>(
+        kernel<<<dim3(tiles, np), kBwdThreads, smem, p.stream>>>(
             t, plan, cfg, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.k, (const __nv_bfloat16*)p.v,
             (const __nv_bfloat16*)p.rel_emb, (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out,
             (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale, p.lengths, p.drop);
