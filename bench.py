@@ -47,7 +47,7 @@ KERNEL_MODEL = {
 # DRAM bytes (read + write) per (batch entry, head) pair of one launch, from the ncu captures summarised
 # under profiles/ (taken at batch 1; every pair is an independent problem, so traffic scales with pairs).
 # An entry is dropped (traffic = null) when its kernel changes after the capture.
-NCU_DRAM_BYTES_PER_PAIR = {"fwd_tc5": 41.25e6 / 8, "bwd_tile": 381.7e6 / 8}  # profiles/tile_kernels_full_cfg4_batch1.md
+NCU_DRAM_BYTES_PER_PAIR = {"fwd_tc5": 41.28e6 / 8, "bwd_tile": 380.1e6 / 8}  # profiles/tile_kernels_full_cfg4_batch1.md
 
 
 def load_peaks():
