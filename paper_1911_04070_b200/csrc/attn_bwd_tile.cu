@@ -44,6 +44,7 @@ struct ChunkPlan {
     int slab_row0[kMaxChunks + 1];  // first reserved partial row of each chunk; [chunks] = rows per tile
     int rel_rows;                   // relation offsets a chunk's products cover (multiple of 16)
     int rel_store;                  // rows kept per chunk in the d_rel partials: k + 2, the most a chunk uses
+    int group;                      // consecutive 64-token tiles one CTA works through (their partial rows are merged)
 };
 
 // Shared-memory layout.  The buffer sizes follow k and are capped so that two CTAs fit an SM (two
@@ -81,7 +82,7 @@ constexpr BwdTileCfg layout_of(int kv_rows, int rel_rows, int qr_stride) {
 constexpr size_t kTwoCtaBytes = 112 * 1024;  // shared memory per CTA up to which two CTAs fit an SM
 
 BwdTileCfg make_bwd_tile_cfg(const TreeParams& t, int chunks) {
-    const size_t tail = (size_t)chunks * (kTileTokens * 8 + 8);
+    const size_t tail = (size_t)chunks * (kTileTokens * 8 + 8 + 5 * 4);  // row ranges, chunk range, group bookkeeping
     const int rel_rows = min(kMaxRelRows, (t.k + 2 + 15) & ~15);
     const int qr_stride = rel_rows - 4 >= t.k + 2 ? rel_rows - 4 : rel_rows + 4;
     int kv_rows = min(kMaxKvRows, (t.kc + 97) & ~15);  // 15 (alignment) + 64 + k + 3 columns at most, rounded up to 16
@@ -133,12 +134,19 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
     int2* bnd = reinterpret_cast<int2*>(delta_s + kTileTokens);
     const int n_left = plan.n_left, n_right = plan.n_right, chunks = n_left + n_right;
     int2* crange = bnd + chunks * kTileTokens;
+    // per chunk, over the tiles of the group done so far: first node of the merged partial rows, last node written,
+    // whether the d_rel partial has been written; and the last two as they were before the current tile
+    int* st_origin = reinterpret_cast<int*>(crange + chunks);
+    int* st_hi = st_origin + chunks;
+    int* st_rel = st_hi + chunks;
+    int* st_old_hi = st_rel + chunks;
+    int* st_rel_old = st_old_hi + chunks;
 
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int kQrStride = cfg.qr_stride, kPStride = cfg.p_stride, kSkewStride = cfg.skew_stride;
     const int rg = w;  // row group: this warp's 16 query rows
     const int g = lane >> 2, c2 = (lane & 3) * 2;
-    const int tile = blockIdx.x, tiles = gridDim.x, t0 = tile * kTileTokens;
+    const int st = blockIdx.x, n_st = gridDim.x;  // group of plan.group consecutive tiles, and how many groups
     const int pair = pair0 + blockIdx.y, b = pair / H, h = pair % H;
     const int N = 2 * t.n - 1;
     const size_t rs = (size_t)H * 64;
@@ -146,6 +154,15 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
     const uint32_t q_u = smem_u32(q_s), g_u = smem_u32(g_s), k_u = smem_u32(k_s), v_u = smem_u32(v_s),
                    r_u = smem_u32(r_s), p_u = smem_u32(p_s), ds_u = smem_u32(ds_s), sk_u = smem_u32(sk_s);
     const float scale_log2e = scale * kLog2e;
+    float* slab_cta = slabs + ((size_t)blockIdx.y * n_st + st) * plan.slab_row0[chunks] * 128;
+    float* drel_cta = drel_part + ((size_t)blockIdx.y * n_st + st) * chunks * plan.rel_store * 64;
+    if (tid < chunks) { st_origin[tid] = 0; st_hi[tid] = -1; st_rel[tid] = 0; }
+
+    // The tiles of the group one after the other.  A later tile adds its partial rows to those an earlier tile
+    // of the same CTA already wrote (read back from L2, same thread order every run), so that the gather finds
+    // one row per node and group instead of one per node and tile.
+    for (int hidx = 0; hidx < plan.group; ++hidx) {
+    const int tile = st * plan.group + hidx, t0 = tile * kTileTokens;
 
     // ---- prologue: Q and dO tiles, out tile (into the K buffer) for the row term, row ranges ----
     for (int idx = tid; idx < kTileTokens * 8; idx += kBwdThreads) {
@@ -189,12 +206,6 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
         if (lane == 0) {
             const int2 u = make_int2(min(a.x, bb.x), max(a.y, bb.y));
             crange[c] = u;
-            if (blockIdx.y == 0 && pair0 == 0) {
-                // empty ranges keep the table monotone over the tiles: left levels are missing for a
-                // prefix of the tiles, right levels for a suffix
-                const int n_l = t.n >> (c >= n_left ? c - n_left : c);
-                tile_range[(size_t)c * tiles + tile] = u.x <= u.y ? u : (c >= n_left ? make_int2(n_l, n_l - 1) : make_int2(0, -1));
-            }
         }
     }
 
@@ -207,8 +218,6 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
     for (int nt = 0; nt < 8; ++nt) { acc_q[nt][0] = acc_q[nt][1] = acc_q[nt][2] = acc_q[nt][3] = 0.f; }
 
     float* qr_w = qr_s + rg * 16 * kQrStride;
-    float* slab_cta = slabs + ((size_t)blockIdx.y * tiles + tile) * plan.slab_row0[chunks] * 128;
-    float* drel_cta = drel_part + ((size_t)blockIdx.y * tiles + tile) * chunks * plan.rel_store * 64;
 
     // A chunk whose node range is wider than the K / V buffers is worked through in sub-blocks of
     // cfg.kv_rows columns; (c, s0) = chunk and first column of the sub-block.  Its length:
@@ -239,6 +248,16 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
         if (tid < kTileTokens) mask_row_bounds(t, t0, tid, n_left, n_right, bnd, len);
     }
     __syncthreads();  // delta and crange are visible; the out tile in the K buffer is consumed
+    if (tid < chunks) {  // group bookkeeping (first read in phase 2, several barriers from here)
+        const int2 u = crange[tid];
+        st_old_hi[tid] = st_hi[tid];
+        st_rel_old[tid] = st_rel[tid];
+        if (u.x <= u.y) {
+            if (st_hi[tid] < 0) st_origin[tid] = u.x;
+            st_hi[tid] = u.y;
+            st_rel[tid] = 1;
+        }
+    }
     stage(0, 0);      // chunk 0 (left level 0 with the self loop) is never empty
     cp_async_commit();
 
@@ -396,11 +415,7 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
         if (last) {
             cn = c + 1;
             sn = 0;
-            while (cn < chunks && crange[cn].x > crange[cn].y) {  // a level no token of the tile reaches: zero d_rel partial
-                float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)cn * plan.rel_store * 64);
-                for (int idx = tid; idx < plan.rel_store * 16; idx += kBwdThreads) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
-                ++cn;
-            }
+            while (cn < chunks && crange[cn].x > crange[cn].y) ++cn;  // a level no token of the tile reaches
         }
         if (cn < chunks) stage(cn, sn);
         cp_async_commit();
@@ -412,11 +427,27 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
             const int hc = job & 1, tile16 = job >> 1;  // channel half, tile
             if (tile16 < n_jt) {
                 const int jt = tile16;
+                // the accumulators start from what an earlier tile of the group left in the partial rows (the loads
+                // fly while the products below run), from zero otherwise
                 float ak[4][4], av[4][4];
+                float* dst_row[2];
+                bool row_ok[2];
 #pragma unroll
-                for (int nt = 0; nt < 4; ++nt) {
-                    ak[nt][0] = ak[nt][1] = ak[nt][2] = ak[nt][3] = 0.f;
-                    av[nt][0] = av[nt][1] = av[nt][2] = av[nt][3] = 0.f;
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int m = base + jt * 16 + g + hh * 8;
+                    row_ok[hh] = m >= cr.x && m <= cr.y;
+                    dst_row[hh] = slab_cta + (size_t)(plan.slab_row0[c] + m - st_origin[c]) * 128 + hc * 32 + c2;
+                    const bool add = row_ok[hh] && m <= st_old_hi[c];
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt) {
+                        float2 xk = make_float2(0.f, 0.f), xv = xk;
+                        if (add) {
+                            xk = *reinterpret_cast<const float2*>(dst_row[hh] + nt * 8);
+                            xv = *reinterpret_cast<const float2*>(dst_row[hh] + 64 + nt * 8);
+                        }
+                        ak[nt][hh * 2] = xk.x; ak[nt][hh * 2 + 1] = xk.y;
+                        av[nt][hh * 2] = xv.x; av[nt][hh * 2 + 1] = xv.y;
+                    }
                 }
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
@@ -436,21 +467,29 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
                 }
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
-                    const int m = base + jt * 16 + g + hh * 8;
-                    if (m >= cr.x && m <= cr.y) {
-                        float* dst = slab_cta + (size_t)(plan.slab_row0[c] + m - cr.x) * 128 + hc * 32 + c2;
+                    if (row_ok[hh]) {
 #pragma unroll
                         for (int nt = 0; nt < 4; ++nt) {
-                            *reinterpret_cast<float2*>(dst + nt * 8) = make_float2(ak[nt][hh * 2], ak[nt][hh * 2 + 1]);
-                            *reinterpret_cast<float2*>(dst + 64 + nt * 8) = make_float2(av[nt][hh * 2], av[nt][hh * 2 + 1]);
+                            *reinterpret_cast<float2*>(dst_row[hh] + nt * 8) = make_float2(ak[nt][hh * 2], ak[nt][hh * 2 + 1]);
+                            *reinterpret_cast<float2*>(dst_row[hh] + 64 + nt * 8) = make_float2(av[nt][hh * 2], av[nt][hh * 2 + 1]);
                         }
                     }
                 }
             } else {
                 const int ot = tile16 - n_jt;
                 float ar[4][4];
+                const bool add = st_rel_old[c] != 0;  // an earlier tile of the group wrote this chunk's partial: start from it
 #pragma unroll
-                for (int nt = 0; nt < 4; ++nt) { ar[nt][0] = ar[nt][1] = ar[nt][2] = ar[nt][3] = 0.f; }
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int o = ot * 16 + g + hh * 8;
+                    const float* src = drel_cta + ((size_t)c * plan.rel_store + o) * 64 + hc * 32 + c2;
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt) {
+                        float2 x = make_float2(0.f, 0.f);
+                        if (add && o < plan.rel_store) x = *reinterpret_cast<const float2*>(src + nt * 8);
+                        ar[nt][hh * 2] = x.x; ar[nt][hh * 2 + 1] = x.y;
+                    }
+                }
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
                     uint32_t a[4];
@@ -491,6 +530,22 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
         const int row = r0 + (idx >> 3), ch = idx & 7;
         *reinterpret_cast<uint4*>(dq + boff + (size_t)(t0 + row) * rs + ch * 8) =
             *reinterpret_cast<const uint4*>(q_s + tile_off(row, ch));
+    }
+    __syncthreads();  // the Q tile is free for the next tile of the group
+    }  // tiles of the group
+
+    // chunks no tile of the group reached: zero d_rel partial; the group's ranges for the gather
+    for (int c = 0; c < chunks; ++c) {
+        if (st_rel[c]) continue;
+        float4* z = reinterpret_cast<float4*>(drel_cta + (size_t)c * plan.rel_store * 64);
+        for (int idx = tid; idx < plan.rel_store * 16; idx += kBwdThreads) z[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    if (blockIdx.y == 0 && pair0 == 0 && tid < chunks) {
+        // empty ranges keep the table monotone over the groups: left levels are missing for a prefix of the
+        // groups, right levels for a suffix
+        const int n_l = t.n >> (tid >= n_left ? tid - n_left : tid);
+        tile_range[(size_t)tid * n_st + st] = st_hi[tid] >= 0 ? make_int2(st_origin[tid], st_hi[tid])
+                                                              : (tid >= n_left ? make_int2(n_l, n_l - 1) : make_int2(0, -1));
     }
 }
 
@@ -600,11 +655,13 @@ size_t pass_bytes() {
 ChunkPlan make_plan(const TreeParams& t) {
     ChunkPlan p{};
     context_levels(t, &p.n_left, &p.n_right);
+    p.group = t.n >= 2 * kTileTokens ? 2 : 1;
+    const int span = p.group * kTileTokens;  // tokens whose partial rows are merged
     int at = 0;
     for (int c = 0; c < p.n_left + p.n_right; ++c) {
         const int level = c >= p.n_left ? c - p.n_left : c;
         p.slab_row0[c] = at;
-        at += (kTileTokens >> level) + t.kc + 3;  // upper bound of a tile's union range at this level
+        at += (span >> level) + t.kc + 3;  // upper bound of the group's union range at this level
     }
     p.slab_row0[p.n_left + p.n_right] = at;
     p.rel_rows = (t.k + 2 + 15) & ~15;
@@ -613,7 +670,7 @@ ChunkPlan make_plan(const TreeParams& t) {
 }
 
 TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, int B, int H, void* base) {
-    const int chunks = plan.n_left + plan.n_right, tiles = t.n / kTileTokens;
+    const int chunks = plan.n_left + plan.n_right, tiles = t.n / (kTileTokens * plan.group);  // groups of tiles
     const size_t per_pair = ((size_t)tiles * ((size_t)plan.slab_row0[chunks] * 128 + (size_t)chunks * plan.rel_store * 64) +
                              bwd_span_slab_floats(t, 1) + bwd_span_ext_floats(t, 1)) * sizeof(float);
     TileWorkspace w;
@@ -649,7 +706,7 @@ size_t bwd_tile_workspace_bytes(const bpt_graph& g, int B, int H) {
 bpt_status launch_bwd_tile(const AttnProblem& p) {
     const TreeParams& t = p.tree;
     const ChunkPlan plan = make_plan(t);
-    const int chunks = plan.n_left + plan.n_right, tiles = t.n / kTileTokens, N = 2 * t.n - 1;
+    const int chunks = plan.n_left + plan.n_right, tiles = t.n / (kTileTokens * plan.group), N = 2 * t.n - 1;  // tiles: groups
     const TileWorkspace ws = carve_tile(t, plan, p.B, p.H, p.workspace);
     const BwdTileCfg cfg = make_bwd_tile_cfg(t, chunks);
     const size_t smem = cfg.bytes;
