@@ -17,7 +17,15 @@
  * `cuda_stream` (a cudaStream_t passed as void*, NULL = legacy default stream) and
  * return without synchronising.  Nothing is allocated or kept between calls, so the attention calls
  * (bpt_attn_fwd / bpt_attn_bwd and their _varlen, _ex, _rows forms) can be captured in a CUDA graph.
+ * The library reads no environment variable and keeps no process-wide setting (the one exception,
+ * the benchmark trace, is described at bpt_trace_begin).
  * Argument errors are detected on the host before anything is launched.
+ *
+ * Device-side failure report.  A non-empty attention workspace begins with a 256-byte status block
+ * that every attention call clears on its stream before its kernels run.  Kernels that wait on
+ * hardware barriers (the tensor-memory kernels) bound every wait to about a second; if one expires
+ * the kernel winds down, the results of the call are invalid and BPT_ERR_TIMEOUT is stored in the
+ * block.  bpt_check reads it.
  */
 #ifndef BPT_H
 #define BPT_H
@@ -31,8 +39,9 @@ extern "C" {
 
 typedef enum {
     BPT_OK = 0,
-    BPT_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, n not a power of two, ... */
-    BPT_ERR_UNSUPPORTED = 2,  /* head size / dtype / range the kernels do not cover        */
+    BPT_ERR_INVALID_ARG = 1,  /* null pointer, non-positive size, unknown flag, ...          */
+    BPT_ERR_UNSUPPORTED = 2,  /* head size / dtype / range the kernels do not cover; n not  */
+                              /* a power of two                                             */
     BPT_ERR_WORKSPACE = 3,    /* workspace missing or smaller than the size query says      */
     BPT_ERR_CUDA = 4,         /* a CUDA runtime call or launch failed                       */
     BPT_ERR_TIMEOUT = 5,      /* a bounded device-side wait expired (see bpt_attn_fwd)      */
@@ -45,8 +54,9 @@ enum {
     BPT_BIDIR = 0,      /* contextual edges from both sides (Sec. 3.2.2)                          */
     BPT_LEFT_ONLY = 1,  /* only the left context, for autoregressive use (Sec. 4.2); self and      */
                         /* affiliated edges are kept                                               */
-    BPT_MODE_PAD = 0,   /* default: k nodes per level plus the extra node that aligns the next     */
-                        /* level with a whole parent ("when the index p_l+k-1 is odd...", 3.2.2)   */
+    BPT_MODE_PAD = 0,   /* default: k nodes per level plus the alignment node of Sec. 3.2.2 -- one  */
+                        /* more when the level's last node is a left child, so that the next level  */
+                        /* starts on a whole parent                                                 */
     BPT_MODE_ALG1 = 2   /* Algorithm 1 taken literally: exactly k nodes per level, no extra node   */
 };
 
@@ -77,8 +87,9 @@ typedef struct {
  * Sec. 3.2: 2n-1 nodes; per token a self loop (Algorithm 1, N <- {u}), k (or k+1
  * with the pad rule) contextual nodes per level and side, fine to coarse; per span
  * one affiliated edge from every token it contains.
- * Requires n a power of two, 2 <= n <= 2^20, 1 <= k <= 2^20.  `out` is a host pointer.
- * Errors: INVALID_ARG, UNSUPPORTED (range), OVERFLOW (E >= 2^31).
+ * Requires n a power of two (Sec. 3.2.1 builds a perfect binary tree; shorter sequences are served
+ * by the length arguments of the attention calls), 2 <= n <= 2^20, 1 <= k <= 2^20.  `out` is a host pointer.
+ * Errors: INVALID_ARG, UNSUPPORTED (range, n not a power of two), OVERFLOW (E >= 2^31).
  */
 bpt_status bpt_graph_dims_query(int32_t n, int32_t k, uint32_t flags, bpt_graph_dims* out);
 
@@ -101,13 +112,26 @@ bpt_status bpt_build_graph(const bpt_graph_dims* dims, int32_t* row_ptr, int32_t
 
 /*
  * Bytes of device workspace bpt_attn_fwd (backward == 0) or bpt_attn_bwd
- * (backward != 0) needs for this problem; 0 on invalid arguments.  Host only.
- * The tiled backward keeps partial gradient rows of as many (batch entry, head) pairs as fit
- * 10 GiB and works through larger problems in passes; BPT_BWD_PASS_MB in the environment (read
- * once per process) sets another cap in MiB, trading workspace for passes.  The same sizes serve
- * the _varlen and _ex forms.
+ * (backward != 0) should be given for this problem; 0 on invalid arguments.  Host only.
+ * The same sizes serve the _varlen and _ex forms.
+ *
+ * The backward accepts any workspace of at least bpt_attn_bwd_min_workspace_bytes: where its
+ * kernels keep per-(batch entry, head) scratch they work through the pairs in passes, as many pairs
+ * per pass as the given bytes hold (the size returned here plans at most 10 GiB per pass).  dq, dk
+ * and dv do not depend on the number of passes; d_rel is summed pass by pass, in a fixed order
+ * for a given workspace size.
  */
 size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype, int backward);
+size_t bpt_attn_bwd_min_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype);
+
+/*
+ * Waits for `cuda_stream` and reports what the last attention call that used `workspace` (device
+ * pointer, the one passed to that call; NULL is allowed and reports BPT_OK) left in the status
+ * block: BPT_OK, or BPT_ERR_TIMEOUT when a bounded device-side wait expired and the call's results
+ * are invalid.  BPT_ERR_CUDA when the synchronisation or the copy fails.  Host-synchronous: not for
+ * use inside a stream capture.
+ */
+bpt_status bpt_check(const void* workspace, void* cuda_stream);
 
 /*
  * Forward graph self-attention with relative positions (Sec. 3.4 equation, built on
@@ -119,12 +143,7 @@ size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_
  * `scale` is explicit (the paper divides by sqrt(d); callers pass 1/sqrt(d)).
  * d must be 32 or 64.  `g` is a host pointer to a struct of device pointers.
  * `workspace` may be NULL when the size query returns 0.
- * Device-side failure report: the kernels that wait on hardware barriers (tensor-memory forward)
- * bound every wait to about a second; if one expires the kernel winds down, the results are
- * invalid and BPT_ERR_TIMEOUT is stored in the 32-bit word at workspace + (size query) - 256,
- * which the call never clears: zero it before the call if you want to read it afterwards
- * (after synchronising the stream).
- * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA; device-side: see bpt_check.
  */
 bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                         const void* q, const void* k, const void* v, const void* rel_emb, float scale,
@@ -185,12 +204,19 @@ bpt_status bpt_attn_bwd_varlen(const bpt_graph* g, int32_t B, int32_t H, int32_t
  * Philox4x32 with 10 rounds, key = (low, high) word of the seed, counter = (destination, source,
  * batch entry * H + head, 0x42505431), edge kept iff the first output word >= floor(dropout_p * 2^32).
  * The backward rebuilds it from the same options (nothing is stored); pass the options the forward had.
- * `opt` is a host pointer; NULL means no lengths and no dropout.  dropout_p outside [0, 1): INVALID_ARG.
+ * `path` picks the kernels of the token rows where the tiled tensor-core path applies (bf16, head
+ * size 64, n >= 64, k <= 64): BPT_PATH_AUTO lets the library choose by k; BPT_PATH_MMA forces the
+ * warp-level (mma.sync) kernels, BPT_PATH_TC5 the tensor-memory (tcgen05) kernels wherever they cover
+ * the shape -- for comparison runs and tests.  Other values: INVALID_ARG.
+ * `opt` is a host pointer; NULL means no lengths, no dropout, automatic path.  dropout_p outside
+ * [0, 1): INVALID_ARG.
  */
+enum { BPT_PATH_AUTO = 0, BPT_PATH_MMA = 1, BPT_PATH_TC5 = 2 };
 typedef struct {
     const int32_t* lengths; /* device [B] or NULL */
     float dropout_p;
     uint64_t dropout_seed;
+    uint32_t path;          /* BPT_PATH_* */
 } bpt_attn_options;
 
 bpt_status bpt_attn_fwd_ex(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
@@ -230,13 +256,19 @@ bpt_status bpt_attn_fwd_rows(const bpt_graph* g, int32_t B, int32_t H, int32_t d
  * Same arguments, results and errors as bpt_attn_bwd, minus the workspace: the scratch
  * is a 32 MiB array that lives inside the library's device image (every GPU that loads
  * the library carries it until the process exits).  bpt_static_scratch_bytes() returns
- * that limit; a problem whose bpt_attn_workspace_bytes(..., backward = 1) exceeds it is
+ * that limit.  The backward fits its passes to the array (fewer (batch entry, head) pairs
+ * per pass than with a large workspace, same results for dq, dk, dv); only a problem whose
+ * bpt_attn_bwd_min_workspace_bytes exceeds the limit -- one pair alone does not fit -- is
  * refused with BPT_ERR_SCRATCH_LIMIT before anything is launched (use bpt_attn_bwd with
  * your own workspace then).  The call itself performs no cudaMalloc / cudaFree and calls
  * no allocating library routine.
  *
  * The first call on each device looks up the array's device address (with that device
- * current); make that first call outside of any stream capture.  All calls on a device
+ * current); make that first call outside of any stream capture.  The CUDA runtime loads the
+ * part of the library that holds the array at that first look-up, and that is when the
+ * driver sets the 32 MiB aside: a process that hands the rest of the device to a pool of its
+ * own should make one call (any small problem) during start-up, before the pool takes the
+ * memory.  All calls on a device
  * share the one array, and it keeps whatever the previous call left in it: the backward
  * overwrites every part before reading it, so nothing needs clearing, but two calls whose
  * GPU work overlaps (different streams, or different threads) would race on it -- keep
@@ -261,6 +293,17 @@ bpt_status bpt_attn_bwd_static_scratch(const bpt_graph* g, int32_t B, int32_t H,
  */
 bpt_status bpt_trace_begin(int32_t capacity, void* cuda_stream);
 bpt_status bpt_trace_end(int32_t* n_marks, float* ms, const char** names, int32_t capacity);
+
+/*
+ * Test hook for the failure report (no counterpart in the paper): launches one tiny kernel in which
+ * one thread waits, for at most `limit_cycles` clock cycles (1 .. 2^31), on a hardware barrier that
+ * expects one arrival.  With arrive == 0 nobody arrives: the wait runs out, the kernel stores
+ * BPT_ERR_TIMEOUT in the status block at `workspace` (device, >= 256 bytes, cleared first) and ends --
+ * exactly the give-up path of the tensor-memory kernels; with arrive != 0 the thread arrives itself
+ * and the block stays clear.  Nothing faults or hangs either way.  Read the outcome with bpt_check.
+ * Errors: INVALID_ARG, CUDA.
+ */
+bpt_status bpt_selftest_wait_timeout(void* workspace, int64_t limit_cycles, int32_t arrive, void* cuda_stream);
 
 /* Static description of a status code (host). */
 const char* bpt_status_str(bpt_status s);

@@ -16,11 +16,13 @@ LIB_PATH = os.path.join(_HERE, "libbpt.so")
 
 BPT_BIDIR, BPT_LEFT_ONLY, BPT_MODE_PAD, BPT_MODE_ALG1 = 0, 1, 0, 2
 BPT_F32, BPT_BF16 = 0, 1
+BPT_PATH_AUTO, BPT_PATH_MMA, BPT_PATH_TC5 = 0, 1, 2
 
 EXPORTS = ("bpt_graph_dims_query", "bpt_build_graph", "bpt_attn_workspace_bytes", "bpt_attn_fwd",
            "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end",
            "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch", "bpt_attn_fwd_varlen", "bpt_attn_bwd_varlen",
-           "bpt_attn_fwd_ex", "bpt_attn_bwd_ex", "bpt_attn_fwd_rows")
+           "bpt_attn_fwd_ex", "bpt_attn_bwd_ex", "bpt_attn_fwd_rows", "bpt_attn_bwd_min_workspace_bytes", "bpt_check",
+           "bpt_selftest_wait_timeout")
 
 
 class BptError(RuntimeError):
@@ -42,8 +44,13 @@ class GraphStruct(ctypes.Structure):
 
 
 class AttnOptions(ctypes.Structure):
-    _fields_ = [("lengths", ctypes.c_void_p), ("dropout_p", ctypes.c_float), ("dropout_seed", ctypes.c_uint64)]
+    _fields_ = [("lengths", ctypes.c_void_p), ("dropout_p", ctypes.c_float), ("dropout_seed", ctypes.c_uint64),
+                ("path", ctypes.c_uint32)]
 
+
+# When set, the autograd wrapper in layer.py asks bpt_check after every attention call (a stream
+# synchronisation per call): for debugging; training loops normally check once per step.
+CHECK_DEVICE_STATUS = False
 
 _lib = None
 
@@ -63,6 +70,12 @@ def load_library() -> ctypes.CDLL:
         lib.bpt_build_graph.argtypes = [ctypes.POINTER(GraphDims), vp, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(GraphStruct)]
         lib.bpt_attn_workspace_bytes.restype = sz
         lib.bpt_attn_workspace_bytes.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, ctypes.c_int]
+        lib.bpt_attn_bwd_min_workspace_bytes.restype = sz
+        lib.bpt_attn_bwd_min_workspace_bytes.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int]
+        lib.bpt_check.restype = ctypes.c_int
+        lib.bpt_check.argtypes = [vp, vp]
+        lib.bpt_selftest_wait_timeout.restype = ctypes.c_int
+        lib.bpt_selftest_wait_timeout.argtypes = [vp, ctypes.c_int64, i32, vp]
         lib.bpt_attn_fwd.restype = ctypes.c_int
         lib.bpt_attn_fwd.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
                                      vp, vp, vp, sz, vp]
@@ -171,6 +184,26 @@ def bpt_attn_workspace_bytes(g: Graph, B: int, H: int, d: int, dtype_code: int, 
     return int(load_library().bpt_attn_workspace_bytes(ctypes.byref(g.c), B, H, d, dtype_code, int(backward)))
 
 
+def bpt_attn_bwd_min_workspace_bytes(g: Graph, B: int, H: int, d: int, dtype_code: int) -> int:
+    """The smallest workspace bpt_attn_bwd accepts (it then works through the problem in more passes)."""
+    return int(load_library().bpt_attn_bwd_min_workspace_bytes(ctypes.byref(g.c), B, H, d, dtype_code))
+
+
+def bpt_check(workspace) -> int:
+    """Waits for the current stream and returns the status the last attention call left in `workspace`
+    (0 = ok, 5 = a bounded device-side wait expired: that call's results are invalid)."""
+    dev = torch.cuda.current_device() if workspace is None else workspace.device
+    with torch.cuda.device(dev):
+        return int(load_library().bpt_check(_ptr(workspace), _stream()))
+
+
+def bpt_selftest_wait_timeout(workspace, limit_cycles: int, arrive: bool):
+    """Launches the library's wait self-test (see include/bpt.h); read the outcome with bpt_check."""
+    with torch.cuda.device(workspace.device):
+        _check(load_library().bpt_selftest_wait_timeout(_ptr(workspace), int(limit_cycles), int(arrive), _stream()),
+               "bpt_selftest_wait_timeout")
+
+
 def _check_layout(g: Graph, q, *same):
     if q.dim() != 4 or q.shape[1] != g.n_nodes:
         raise ValueError("expected [B, n_nodes=%d, H, d], got %s" % (g.n_nodes, tuple(q.shape)))
@@ -190,10 +223,11 @@ def _check_lengths(lengths, q):
 
 
 def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, workspace=None, lengths=None,
-                 dropout_p: float = 0.0, dropout_seed: int = 0):
+                 dropout_p: float = 0.0, dropout_seed: int = 0, path: int = BPT_PATH_AUTO):
     """Returns (out [B,N,H,d], lse [B,N,H] fp32).  With `lengths` (int32 [B] on the device) batch entry b
     has lengths[b] real tokens; with dropout_p > 0 the attention weights are dropped (mask defined by
-    dropout_seed); see bpt_attn_fwd_varlen / bpt_attn_fwd_ex in include/bpt.h."""
+    dropout_seed); `path` forces a kernel family; see bpt_attn_fwd_varlen / bpt_attn_fwd_ex in include/bpt.h.
+    A workspace the wrapper allocates itself stays reachable as `out._bpt_workspace` for bpt_check."""
     lib = load_library()
     _check_layout(g, q, k, v)
     B, N, H, d = q.shape
@@ -207,10 +241,11 @@ def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, w
         if workspace is None and need:
             workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
         ws_n = 0 if workspace is None else workspace.numel()
-        if dropout_p:
+        out._bpt_workspace = workspace
+        if dropout_p or path:
             if lengths is not None:
                 _check_lengths(lengths, q)
-            opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed))
+            opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed), int(path))
             _check(lib.bpt_attn_fwd_ex(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
                                        float(scale), ctypes.byref(opt), _ptr(out), _ptr(lse), _ptr(workspace), ws_n,
                                        _stream()), "bpt_attn_fwd_ex")
@@ -226,9 +261,11 @@ def bpt_attn_fwd(g: Graph, q, k, v, rel_emb, scale: float, out=None, lse=None, w
 
 
 def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, workspace=None,
-                 dq=None, dk=None, dv=None, d_rel=None, lengths=None, dropout_p: float = 0.0, dropout_seed: int = 0):
+                 dq=None, dk=None, dv=None, d_rel=None, lengths=None, dropout_p: float = 0.0, dropout_seed: int = 0,
+                 path: int = BPT_PATH_AUTO):
     """Returns (dq, dk, dv [B,N,H,d], d_rel [n_rel, d] fp32).  `lengths`, `dropout_p`, `dropout_seed` as for
-    bpt_attn_fwd (pass what the forward had)."""
+    bpt_attn_fwd (pass what the forward had).  A workspace the wrapper allocates itself stays reachable as
+    `dq._bpt_workspace` for bpt_check."""
     lib = load_library()
     _check_layout(g, q, k, v, out, d_out)
     B, N, H, d = q.shape
@@ -242,10 +279,11 @@ def bpt_attn_bwd(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, work
         if workspace is None and need:
             workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
         ws_n = 0 if workspace is None else workspace.numel()
-        if dropout_p:
+        dq._bpt_workspace = workspace
+        if dropout_p or path:
             if lengths is not None:
                 _check_lengths(lengths, q)
-            opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed))
+            opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed), int(path))
             _check(lib.bpt_attn_bwd_ex(ctypes.byref(g.c), B, H, d, code, _ptr(q), _ptr(k), _ptr(v), _ptr(rel_emb),
                                        float(scale), ctypes.byref(opt), _ptr(out), _ptr(lse), _ptr(d_out), _ptr(dq),
                                        _ptr(dk), _ptr(dv), _ptr(d_rel), _ptr(workspace), ws_n, _stream()), "bpt_attn_bwd_ex")
@@ -273,21 +311,12 @@ def bpt_attn_fwd_rows(g: Graph, q, k, v, rel_emb, scale: float, rows, out, lse, 
         raise ValueError("rows must be a contiguous int32 tensor [B, n_rows] on the device of q")
     if lengths is not None:
         _check_lengths(lengths, q)
-    opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed))
+    opt = AttnOptions(_ptr(lengths), float(dropout_p), int(dropout_seed), 0)
     with torch.cuda.device(q.device):
         _check(load_library().bpt_attn_fwd_rows(ctypes.byref(g.c), B, H, d, _dtype_code(q), _ptr(q), _ptr(k), _ptr(v),
                                                 _ptr(rel_emb), float(scale), ctypes.byref(opt), _ptr(rows), rows.shape[1],
                                                 _ptr(out), _ptr(lse), _stream()), "bpt_attn_fwd_rows")
     return out, lse
-
-
-def bpt_forward_status(workspace) -> int:
-    """The device-side status word of a forward workspace (0 = ok, 5 = a bounded wait expired), read after a
-    stream synchronisation.  The library never clears it: zero the workspace before the call."""
-    if workspace is None or workspace.numel() < 256:
-        return 0
-    torch.cuda.synchronize(workspace.device)
-    return int(workspace[-256:-252].view(torch.int32).item())
 
 
 def bpt_static_scratch_bytes() -> int:
@@ -297,8 +326,9 @@ def bpt_static_scratch_bytes() -> int:
 def bpt_attn_bwd_static_scratch(g: Graph, q, k, v, rel_emb, scale: float, out, lse, d_out, dq, dk, dv, d_rel):
     """Backward pass that takes its scratch from the library's built-in device array instead
     of a workspace tensor, for callers that are not allowed to allocate device memory.  The
-    caller passes every input and output (this wrapper allocates nothing either); problems
-    above bpt_static_scratch_bytes() raise BptError with status 7.  Calls share the array:
+    caller passes every input and output (this wrapper allocates nothing either); a problem
+    of which one (batch entry, head) pair alone needs more than bpt_static_scratch_bytes() raises
+    BptError with status 7.  Calls share the array:
     keep them ordered on one stream."""
     _check_layout(g, q, k, v, out, d_out, dq, dk, dv)
     B, N, H, d = q.shape

@@ -9,6 +9,7 @@ static bpt_status check_problem(const bpt_graph* g, int32_t B, int32_t H, int32_
     if (dtype != BPT_F32 && dtype != BPT_BF16) return BPT_ERR_INVALID_ARG;
     if (d != 32 && d != 64) return BPT_ERR_UNSUPPORTED;
     TreeParams t;
+    if (g->dims.n >= 2 && (g->dims.n & (g->dims.n - 1)) != 0) return BPT_ERR_UNSUPPORTED;
     if (!tree_params_from_dims(g->dims, &t)) return BPT_ERR_INVALID_ARG;
     if (g->dims.n_nodes != 2 * g->dims.n - 1 || g->dims.n_edges < g->dims.n_nodes || g->dims.n_edges >= INT32_MAX)
         return BPT_ERR_INVALID_ARG;
@@ -16,37 +17,66 @@ static bpt_status check_problem(const bpt_graph* g, int32_t B, int32_t H, int32_
     return BPT_OK;
 }
 
+// Every non-empty workspace starts with a 256-byte status block (first word: 0, or the bpt_status a
+// kernel reported); the launchers get what follows it.
+constexpr size_t kStatusBytes = 256;
+static size_t with_status(size_t inner) { return inner ? inner + kStatusBytes : 0; }
+
 extern "C" size_t bpt_attn_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype, int backward) {
     if (check_problem(g, B, H, d, dtype, false) != BPT_OK) return 0;
-    return backward ? bwd_workspace_bytes(*g, B, H, d, dtype) : fwd_workspace_bytes(*g, B, H, d, dtype);
+    return with_status(backward ? bwd_workspace_bytes(*g, B, H, d, dtype) : fwd_workspace_bytes(*g, B, H, d, dtype));
 }
 
-static bool options_ok(const bpt_attn_options* opt) { return !opt || (opt->dropout_p >= 0.f && opt->dropout_p < 1.f); }
+extern "C" size_t bpt_attn_bwd_min_workspace_bytes(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype) {
+    if (check_problem(g, B, H, d, dtype, false) != BPT_OK) return 0;
+    return with_status(bwd_workspace_bytes(*g, B, H, d, dtype, true));
+}
+
+extern "C" bpt_status bpt_check(const void* workspace, void* cuda_stream) {
+    if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return BPT_ERR_CUDA;
+    if (!workspace) return BPT_OK;
+    int32_t word = 0;
+    if (cudaMemcpy(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return BPT_ERR_CUDA;
+    return word == 0 ? BPT_OK : (word == (int32_t)BPT_ERR_TIMEOUT ? BPT_ERR_TIMEOUT : BPT_ERR_CUDA);
+}
+
+static bool options_ok(const bpt_attn_options* opt) {
+    return !opt || (opt->dropout_p >= 0.f && opt->dropout_p < 1.f && opt->path <= BPT_PATH_TC5);
+}
+
+// Splits the caller's workspace into the status block (cleared on the stream) and the launcher's part.
+static bpt_status take_workspace(AttnProblem& p, void* workspace, size_t workspace_bytes, size_t inner_need) {
+    p.status = nullptr; p.workspace = nullptr; p.workspace_bytes = 0;
+    if (inner_need == 0) return BPT_OK;
+    if (!workspace || workspace_bytes < inner_need + kStatusBytes) return BPT_ERR_WORKSPACE;
+    p.status = static_cast<int*>(workspace);
+    p.workspace = static_cast<char*>(workspace) + kStatusBytes;
+    p.workspace_bytes = workspace_bytes - kStatusBytes;
+    return cudaMemsetAsync(workspace, 0, kStatusBytes, p.stream) == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
+}
 
 static bpt_status attn_fwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                 const void* q, const void* k, const void* v, const void* rel_emb, float scale,
-                                const int32_t* lengths, DropoutParams drop, void* out, float* lse, void* workspace,
+                                const int32_t* lengths, DropoutParams drop, uint32_t path, void* out, float* lse, void* workspace,
                                 size_t workspace_bytes, void* cuda_stream) {
     const bpt_status s = check_problem(g, B, H, d, dtype, false);
     if (s != BPT_OK) return s;
     if (!q || !k || !v || !rel_emb || !out || !lse) return BPT_ERR_INVALID_ARG;
-    const size_t need = fwd_workspace_bytes(*g, B, H, d, dtype);
-    if (need > 0 && (!workspace || workspace_bytes < need)) return BPT_ERR_WORKSPACE;
     AttnProblem p{};
     p.g = g;
     tree_params_from_dims(g->dims, &p.tree);
     p.B = B; p.H = H; p.d = d; p.dtype = dtype;
-    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths; p.drop = drop;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths; p.drop = drop; p.path = path;
     p.out = out; p.lse = lse;
-    p.workspace = workspace; p.workspace_bytes = workspace_bytes;
     p.stream = (cudaStream_t)cuda_stream;
-    return launch_fwd(p);
+    const bpt_status w = take_workspace(p, workspace, workspace_bytes, fwd_workspace_bytes(*g, B, H, d, dtype));
+    return w != BPT_OK ? w : launch_fwd(p);
 }
 
 extern "C" bpt_status bpt_attn_fwd(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                    const void* q, const void* k, const void* v, const void* rel_emb, float scale,
                                    void* out, float* lse, void* workspace, size_t workspace_bytes, void* cuda_stream) {
-    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, make_dropout(0.f, 0), out, lse, workspace, workspace_bytes, cuda_stream);
+    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, make_dropout(0.f, 0), BPT_PATH_AUTO, out, lse, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" bpt_status bpt_attn_fwd_varlen(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
@@ -54,7 +84,7 @@ extern "C" bpt_status bpt_attn_fwd_varlen(const bpt_graph* g, int32_t B, int32_t
                                           const int32_t* lengths, void* out, float* lse, void* workspace,
                                           size_t workspace_bytes, void* cuda_stream) {
     if (!lengths) return BPT_ERR_INVALID_ARG;
-    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, make_dropout(0.f, 0), out, lse, workspace, workspace_bytes, cuda_stream);
+    return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, make_dropout(0.f, 0), BPT_PATH_AUTO, out, lse, workspace, workspace_bytes, cuda_stream);
 }
 
 extern "C" bpt_status bpt_attn_fwd_ex(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
@@ -63,30 +93,29 @@ extern "C" bpt_status bpt_attn_fwd_ex(const bpt_graph* g, int32_t B, int32_t H, 
                                       size_t workspace_bytes, void* cuda_stream) {
     if (!options_ok(opt)) return BPT_ERR_INVALID_ARG;
     return attn_fwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, opt ? opt->lengths : nullptr,
-                         opt ? make_dropout(opt->dropout_p, opt->dropout_seed) : make_dropout(0.f, 0), out, lse, workspace,
-                         workspace_bytes, cuda_stream);
+                         opt ? make_dropout(opt->dropout_p, opt->dropout_seed) : make_dropout(0.f, 0), opt ? opt->path : BPT_PATH_AUTO,
+                         out, lse, workspace, workspace_bytes, cuda_stream);
 }
 
 static bpt_status attn_bwd_impl(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
                                 const void* q, const void* k, const void* v, const void* rel_emb, float scale,
-                                const int32_t* lengths, DropoutParams drop, const void* out, const float* lse, const void* d_out,
+                                const int32_t* lengths, DropoutParams drop, uint32_t path, const void* out, const float* lse, const void* d_out,
                                 void* dq, void* dk, void* dv, float* d_rel,
                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
     const bpt_status s = check_problem(g, B, H, d, dtype, true);
     if (s != BPT_OK) return s;
     if (!q || !k || !v || !rel_emb || !out || !lse || !d_out || !dq || !dk || !dv || !d_rel) return BPT_ERR_INVALID_ARG;
-    const size_t need = bwd_workspace_bytes(*g, B, H, d, dtype);
-    if (need > 0 && (!workspace || workspace_bytes < need)) return BPT_ERR_WORKSPACE;
     AttnProblem p{};
     p.g = g;
     tree_params_from_dims(g->dims, &p.tree);
     p.B = B; p.H = H; p.d = d; p.dtype = dtype;
-    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths; p.drop = drop;
+    p.q = q; p.k = k; p.v = v; p.rel_emb = rel_emb; p.scale = scale; p.lengths = lengths; p.drop = drop; p.path = path;
     p.out = const_cast<void*>(out); p.lse = const_cast<float*>(lse);
     p.d_out = d_out; p.dq = dq; p.dk = dk; p.dv = dv; p.d_rel = d_rel;
-    p.workspace = workspace; p.workspace_bytes = workspace_bytes;
     p.stream = (cudaStream_t)cuda_stream;
-    return launch_bwd(p);
+    // the tiled backward runs with any workspace from the minimum up: fewer pairs per pass with a smaller one
+    const bpt_status w = take_workspace(p, workspace, workspace_bytes, bwd_workspace_bytes(*g, B, H, d, dtype, true));
+    return w != BPT_OK ? w : launch_bwd(p);
 }
 
 extern "C" bpt_status bpt_attn_fwd_rows(const bpt_graph* g, int32_t B, int32_t H, int32_t d, bpt_dtype dtype,
@@ -113,7 +142,7 @@ extern "C" bpt_status bpt_attn_bwd(const bpt_graph* g, int32_t B, int32_t H, int
                                    const void* out, const float* lse, const void* d_out,
                                    void* dq, void* dk, void* dv, float* d_rel,
                                    void* workspace, size_t workspace_bytes, void* cuda_stream) {
-    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, make_dropout(0.f, 0), out, lse, d_out, dq, dk, dv, d_rel,
+    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, nullptr, make_dropout(0.f, 0), BPT_PATH_AUTO, out, lse, d_out, dq, dk, dv, d_rel,
                          workspace, workspace_bytes, cuda_stream);
 }
 
@@ -123,7 +152,7 @@ extern "C" bpt_status bpt_attn_bwd_varlen(const bpt_graph* g, int32_t B, int32_t
                                           void* dq, void* dk, void* dv, float* d_rel,
                                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!lengths) return BPT_ERR_INVALID_ARG;
-    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, make_dropout(0.f, 0), out, lse, d_out, dq, dk, dv, d_rel,
+    return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, lengths, make_dropout(0.f, 0), BPT_PATH_AUTO, out, lse, d_out, dq, dk, dv, d_rel,
                          workspace, workspace_bytes, cuda_stream);
 }
 
@@ -134,8 +163,8 @@ extern "C" bpt_status bpt_attn_bwd_ex(const bpt_graph* g, int32_t B, int32_t H, 
                                       void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (!options_ok(opt)) return BPT_ERR_INVALID_ARG;
     return attn_bwd_impl(g, B, H, d, dtype, q, k, v, rel_emb, scale, opt ? opt->lengths : nullptr,
-                         opt ? make_dropout(opt->dropout_p, opt->dropout_seed) : make_dropout(0.f, 0), out, lse, d_out,
-                         dq, dk, dv, d_rel, workspace, workspace_bytes, cuda_stream);
+                         opt ? make_dropout(opt->dropout_p, opt->dropout_seed) : make_dropout(0.f, 0), opt ? opt->path : BPT_PATH_AUTO,
+                         out, lse, d_out, dq, dk, dv, d_rel, workspace, workspace_bytes, cuda_stream);
 }
 
 // ---------------------------------------------------------------------------------

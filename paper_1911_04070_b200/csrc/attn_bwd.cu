@@ -401,11 +401,11 @@ static bpt_status launch_bwd_rows(const AttnProblem& p) {
 }
 
 bool bwd_tile_eligible(const bpt_graph& g, int d, bpt_dtype dtype);
-size_t bwd_tile_workspace_bytes(const bpt_graph& g, int B, int H);
+size_t bwd_tile_workspace_bytes(const bpt_graph& g, int B, int H, bool minimal);
 bpt_status launch_bwd_tile(const AttnProblem& p);
 
-size_t bwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype) {
-    if (bwd_tile_eligible(g, d, dtype)) return bwd_tile_workspace_bytes(g, B, H);
+size_t bwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype, bool minimal) {
+    if (bwd_tile_eligible(g, d, dtype)) return bwd_tile_workspace_bytes(g, B, H, minimal);
     return carve(g, B, H, d, nullptr).bytes;
 }
 

@@ -18,8 +18,6 @@
 // Nothing is accumulated across CTAs here: bwd_gather_kernel sums, for every source node, the
 // partial rows of the tiles whose range covers it, in tile order (no atomics, fixed order), and
 // drel_sum kernels do the same for the relation table.
-#include <cstdlib>
-
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
 #include "row_map.cuh"
@@ -641,16 +639,9 @@ struct TileWorkspace {
     size_t bytes;
 };
 
-// Partial rows kept per pass over the (batch entry, head) pairs: 10 GiB, or BPT_BWD_PASS_MB from the
-// environment (read once; smaller values trade workspace for more passes).
-size_t pass_bytes() {
-    static const size_t v = [] {
-        const char* e = getenv("BPT_BWD_PASS_MB");
-        const long mb = e ? atol(e) : 0;
-        return mb > 0 ? (size_t)mb << 20 : (size_t)10 << 30;
-    }();
-    return v;
-}
+// Partial rows the size query plans per pass over the (batch entry, head) pairs.  A caller that brings a
+// smaller workspace gets more passes: the launcher fits as many pairs as the given bytes hold.
+constexpr size_t kPassBytes = (size_t)10 << 30;
 
 ChunkPlan make_plan(const TreeParams& t) {
     ChunkPlan p{};
@@ -669,14 +660,10 @@ ChunkPlan make_plan(const TreeParams& t) {
     return p;
 }
 
-TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, int B, int H, void* base) {
+// Carves the workspace for `pairs` (batch entry, head) pairs per pass.
+TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, size_t pairs, void* base) {
     const int chunks = plan.n_left + plan.n_right, tiles = t.n / (kTileTokens * plan.group);  // groups of tiles
-    const size_t per_pair = ((size_t)tiles * ((size_t)plan.slab_row0[chunks] * 128 + (size_t)chunks * plan.rel_store * 64) +
-                             bwd_span_slab_floats(t, 1) + bwd_span_ext_floats(t, 1)) * sizeof(float);
     TileWorkspace w;
-    size_t pairs = pass_bytes() / per_pair;
-    if (pairs < 1) pairs = 1;
-    if (pairs > (size_t)B * H) pairs = (size_t)B * H;
     w.pairs_per_pass = (int)pairs;
     char* c = (char*)base;
     size_t off = 0;
@@ -690,16 +677,30 @@ TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, int B, int 
     return w;
 }
 
+// Pairs per pass: as many as `budget` bytes hold (at least one, at most all).
+size_t pairs_for_budget(const TreeParams& t, const ChunkPlan& plan, int B, int H, size_t budget) {
+    const size_t all = (size_t)B * H;
+    const size_t fixed = carve_tile(t, plan, 0, nullptr).bytes;
+    const size_t per_pair = carve_tile(t, plan, 1, nullptr).bytes - fixed;  // an upper bound: it includes the rounding of one pair
+    size_t pairs = budget > fixed ? (budget - fixed) / per_pair : 0;
+    if (pairs > all) pairs = all;
+    while (pairs < all && carve_tile(t, plan, pairs + 1, nullptr).bytes <= budget) ++pairs;
+    return pairs < 1 ? 1 : pairs;
+}
+
 }  // namespace
 
 bool bwd_tile_eligible(const bpt_graph& g, int d, bpt_dtype dtype) {
     return tile_path(g.dims.n, g.dims.k, d, dtype == BPT_BF16);
 }
 
-size_t bwd_tile_workspace_bytes(const bpt_graph& g, int B, int H) {
+// minimal: the smallest workspace the backward runs with (one pair per pass); otherwise the planned size.
+size_t bwd_tile_workspace_bytes(const bpt_graph& g, int B, int H, bool minimal) {
     TreeParams t;
     tree_params_from_dims(g.dims, &t);
-    return carve_tile(t, make_plan(t), B, H, nullptr).bytes;
+    const ChunkPlan plan = make_plan(t);
+    const size_t pairs = minimal ? 1 : pairs_for_budget(t, plan, B, H, kPassBytes);
+    return carve_tile(t, plan, pairs, nullptr).bytes;
 }
 
 
@@ -707,7 +708,8 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
     const TreeParams& t = p.tree;
     const ChunkPlan plan = make_plan(t);
     const int chunks = plan.n_left + plan.n_right, tiles = t.n / (kTileTokens * plan.group), N = 2 * t.n - 1;  // tiles: groups
-    const TileWorkspace ws = carve_tile(t, plan, p.B, p.H, p.workspace);
+    const TileWorkspace ws = carve_tile(t, plan, pairs_for_budget(t, plan, p.B, p.H, p.workspace_bytes), p.workspace);
+    if (ws.bytes > p.workspace_bytes) return BPT_ERR_WORKSPACE;
     const BwdTileCfg cfg = make_bwd_tile_cfg(t, chunks);
     const size_t smem = cfg.bytes;
     if (smem > 227 * 1024) return BPT_ERR_UNSUPPORTED;

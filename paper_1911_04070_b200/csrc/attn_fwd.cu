@@ -159,30 +159,25 @@ bpt_status launch_fwd_tc5(const AttnProblem& p, int* status);
 size_t fwd_span_workspace_bytes(const TreeParams& t, int B, int H);
 bpt_status launch_fwd_span(const AttnProblem& p);
 
-constexpr size_t kStatusBytes = 256;  // device status word at the end of the forward workspace
-
 static size_t span_ws_bytes(const TreeParams& t, int B, int H) { return (fwd_span_workspace_bytes(t, B, H) + 255) & ~(size_t)255; }
 
 size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype) {
     if (!tile_path(g.dims.n, g.dims.k, d, dtype == BPT_BF16)) return 0;
     TreeParams t;
     tree_params_from_dims(g.dims, &t);
-    return span_ws_bytes(t, B, H) + kStatusBytes;
+    return span_ws_bytes(t, B, H) + 256;  // never empty, so that the status block in front of it exists for the tensor-memory kernel
 }
 
 // Two kernels cover the token rows: the warp-level one (mma.sync, 64-token tiles) and the tensor-memory
 // one (tcgen05 + TMA, 128-token tiles).  The second wins where a chunk holds enough nodes per token to
 // pay for its per-chunk hand-offs (measured at n = 8192: 0.32 against 0.34 ms at k = 64, 0.33 against 0.30 ms at
-// k = 48, 0.34 against 0.26 ms at k = 16; 6 to 12 % faster at k = 64 for n = 4096 .. 65536), so it takes k >= 56.  BPT_FWD_TOKENS=tc5 / =mma in the environment forces one of them for comparison runs.
-static bool want_tc5(int k) {
-    static const int forced = [] { const char* e = getenv("BPT_FWD_TOKENS"); return !e ? 0 : (e[0] == 't' ? 1 : (e[0] == 'm' ? 2 : 0)); }();
-    return forced == 1 || (forced == 0 && k >= 56);
-}
+// k = 48, 0.34 against 0.26 ms at k = 16; 6 to 12 % faster at k = 64 for n = 4096 .. 65536), so it takes k >= 56.
+// bpt_attn_options.path forces one of them for comparison runs.
+static bool want_tc5(int k, uint32_t path) { return path == BPT_PATH_TC5 || (path == BPT_PATH_AUTO && k >= 56); }
 
 bpt_status launch_fwd(const AttnProblem& p) {
     if (tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16)) {  // token rows and span rows on the tensor cores
-        int* status = reinterpret_cast<int*>(static_cast<char*>(p.workspace) + span_ws_bytes(p.tree, p.B, p.H));
-        const bpt_status s = (want_tc5(p.tree.k) && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, status) : launch_fwd_tile(p);
+        const bpt_status s = (want_tc5(p.tree.k, p.path) && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, p.status) : launch_fwd_tile(p);
         return s != BPT_OK ? s : launch_fwd_span(p);
     }
     const int row0 = 0, nrows = p.g->dims.n_nodes;

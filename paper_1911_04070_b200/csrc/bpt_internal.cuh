@@ -30,8 +30,10 @@ struct AttnProblem {
     const void* d_out;
     void *dq, *dk, *dv;
     float* d_rel;
-    void* workspace;
+    void* workspace;         // past the status block
     size_t workspace_bytes;
+    int* status;             // device status word (first word of the caller's workspace), or nullptr without a workspace
+    uint32_t path;           // BPT_PATH_*: which token-row kernels the tiled path takes
     cudaStream_t stream;
 };
 
@@ -39,7 +41,8 @@ struct AttnProblem {
 void trace_mark(cudaStream_t st, const char* name);
 
 size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype);
-size_t bwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype);
+// minimal: the least the backward accepts (the tiled path then takes one (batch entry, head) pair per pass)
+size_t bwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dtype, bool minimal = false);
 bpt_status launch_fwd(const AttnProblem& p);
 bpt_status launch_fwd_row_list(const AttnProblem& p, const int32_t* rows, int n_rows);
 bpt_status launch_bwd(const AttnProblem& p);

@@ -255,6 +255,7 @@ extern "C" bpt_status bpt_graph_dims_query(int32_t n, int32_t k, uint32_t flags,
     if (!out) return BPT_ERR_INVALID_ARG;
     if (flags & ~(uint32_t)(BPT_LEFT_ONLY | BPT_MODE_ALG1)) return BPT_ERR_INVALID_ARG;
     TreeParams t;
+    if (n >= 2 && (n & (n - 1)) != 0) return BPT_ERR_UNSUPPORTED;  // the tree of Sec. 3.2.1 is perfect: shorter sequences go through the length arguments
     if (!make_params(n, k, flags, &t)) return BPT_ERR_INVALID_ARG;
     if (n > (1 << 20) || k > (1 << 20)) return BPT_ERR_UNSUPPORTED;
     int64_t e = (int64_t)n * t.L;

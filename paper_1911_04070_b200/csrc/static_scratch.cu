@@ -41,7 +41,9 @@ extern "C" bpt_status bpt_attn_bwd_static_scratch(const bpt_graph* g, int32_t B,
                                                   float scale, const void* out, const float* lse, const void* d_out,
                                                   void* dq, void* dk, void* dv, float* d_rel, void* cuda_stream) {
     if (!g) return BPT_ERR_INVALID_ARG;
-    const size_t need = bpt_attn_workspace_bytes(g, B, H, d, dtype, 1);
+    // The tiled backward works through the (batch entry, head) pairs in as many passes as the array's size
+    // dictates; only a problem whose single pair does not fit is refused.
+    const size_t need = bpt_attn_bwd_min_workspace_bytes(g, B, H, d, dtype);
     if (need > kStaticScratchBytes) return BPT_ERR_SCRATCH_LIMIT;
     void* scratch = nullptr;
     const bpt_status s = device_scratch(&scratch);

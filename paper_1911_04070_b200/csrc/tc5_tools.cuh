@@ -52,15 +52,17 @@ __device__ __forceinline__ void mbar_init(uint32_t mbar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
-// Waits for the phase with the given parity; gives up (returns false) after about a second.
-__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity) {
+// Waits for the phase with the given parity; gives up (returns false) after `limit` clock cycles
+// (default: about a second).
+constexpr long long kWaitCycles = 1ll << 31;
+__device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, long long limit = kWaitCycles) {
     const long long start = clock64();
     for (;;) {
         uint32_t ok;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
                      : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
         if (ok) return true;
-        if (clock64() - start > (1ll << 31)) return false;
+        if (clock64() - start > limit) return false;
     }
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t mbar) {

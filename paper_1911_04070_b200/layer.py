@@ -23,6 +23,8 @@ class _GraphSelfAttention(torch.autograd.Function):
         q, k, v, rel_emb = q.contiguous(), k.contiguous(), v.contiguous(), rel_emb.contiguous()
         out, lse = binding.bpt_attn_fwd(g, q, k, v, rel_emb, scale, lengths=lengths, dropout_p=dropout_p,
                                         dropout_seed=dropout_seed)
+        if binding.CHECK_DEVICE_STATUS and binding.bpt_check(getattr(out, "_bpt_workspace", None)):
+            raise RuntimeError("graph self-attention forward: a device-side wait timed out, results are invalid")
         ctx.save_for_backward(q, k, v, rel_emb, out, lse)
         ctx.g, ctx.scale, ctx.lengths, ctx.drop = g, scale, lengths, (dropout_p, dropout_seed)
         return out
@@ -32,6 +34,8 @@ class _GraphSelfAttention(torch.autograd.Function):
         q, k, v, rel_emb, out, lse = ctx.saved_tensors
         dq, dk, dv, d_rel = binding.bpt_attn_bwd(ctx.g, q, k, v, rel_emb, ctx.scale, out, lse, d_out.contiguous(),
                                                  lengths=ctx.lengths, dropout_p=ctx.drop[0], dropout_seed=ctx.drop[1])
+        if binding.CHECK_DEVICE_STATUS and binding.bpt_check(getattr(dq, "_bpt_workspace", None)):
+            raise RuntimeError("graph self-attention backward: a device-side wait timed out, results are invalid")
         return dq, dk, dv, d_rel.to(rel_emb.dtype), None, None, None, None, None
 
 

@@ -41,7 +41,7 @@ def test_dims_query_matches_closed_forms(lib):
 
 def test_argument_errors(lib):
     from paper_1911_04070_b200 import binding
-    for args, status in [((7, 1, 0), 1), ((8, 0, 0), 1), ((8, 1, 8), 1), ((1, 1, 0), 1), ((1 << 21, 1, 0), 2),
+    for args, status in [((7, 1, 0), 2), ((48, 4, 0), 2), ((8, 0, 0), 1), ((8, 1, 8), 1), ((1, 1, 0), 1), ((1 << 21, 1, 0), 2),
                          ((8, (1 << 20) + 1, 0), 2)]:
         with pytest.raises(binding.BptError) as ei:
             binding.bpt_graph_dims_query(*args)
@@ -52,6 +52,8 @@ def test_argument_errors(lib):
     assert lib.bpt_attn_workspace_bytes(ctypes.byref(g), 1, 1, 64, 0, 0) == 0
     assert lib.bpt_attn_fwd(None, 1, 1, 64, 0, None, None, None, None, 1.0, None, None, None, 0, None) == 1
     assert binding.status_str(3) == "workspace missing or too small"
+    assert lib.bpt_attn_bwd_min_workspace_bytes(ctypes.byref(g), 1, 1, 64, 0) == 0
+    assert lib.bpt_selftest_wait_timeout(None, 1000, 0, None) == 1      # refused on the host: nothing is launched
 
 
 def test_oracle_edge_count_agrees_with_host_query(lib):

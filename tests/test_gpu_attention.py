@@ -17,9 +17,11 @@ def _np(t):
     return t.detach().float().cpu().numpy().astype(np.float64)
 
 
-def run_case(n, k, flags, B, H, d, bf16, seed, std_qkv, backward=True, oracle_batches=None, std_rel=0.02):
+def run_case(n, k, flags, B, H, d, bf16, seed, std_qkv, backward=True, oracle_batches=None, std_rel=0.02,
+             path=0, bwd_workspace_frac=None):
     """Runs the library on the full problem and the oracle (C twin) on the same inputs.
-    Returns nothing; asserts parity."""
+    Returns nothing; asserts parity.  path: BPT_PATH_* forced on both passes; bwd_workspace_frac: give the
+    backward that fraction of the planned workspace (at least the minimum), so that it runs in passes."""
     import torch
     from oracle import ctwin
     from paper_1911_04070_b200 import binding, synth
@@ -29,15 +31,21 @@ def run_case(n, k, flags, B, H, d, bf16, seed, std_qkv, backward=True, oracle_ba
     scale = 1.0 / np.sqrt(d)
     g = binding.bpt_build_graph(n, k, flags, device="cuda:0", with_transpose=backward)
     t = _torch_inputs(x, bf16)
-    out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale)
-    torch.cuda.synchronize()
+    out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, path=path)
+    assert binding.bpt_check(out._bpt_workspace) == 0
     o_ref, lse_ref = ctwin.attn_fwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], scale)
     assert_close("out", _np(out), o_ref, tol)
     assert_close("lse", _np(lse), lse_ref, tol)
     if not backward:
         return
-    dq, dk, dv, dr = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"])
-    torch.cuda.synchronize()
+    ws = None
+    if bwd_workspace_frac is not None:
+        code = binding.BPT_BF16 if bf16 else binding.BPT_F32
+        planned = binding.bpt_attn_workspace_bytes(g, B, H, d, code, True)
+        least = binding.bpt_attn_bwd_min_workspace_bytes(g, B, H, d, code)
+        ws = torch.empty(max(int(planned * bwd_workspace_frac), least), dtype=torch.uint8, device="cuda:0")
+    dq, dk, dv, dr = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"], workspace=ws, path=path)
+    assert binding.bpt_check(dq._bpt_workspace) == 0
     L, W = ref.L, k + 1
     first_anc = 1 + 2 * L * W
     # (1) against the exact gradient: max-norm relative error
@@ -54,8 +62,8 @@ def run_case(n, k, flags, B, H, d, bf16, seed, std_qkv, backward=True, oracle_ba
     assert_close("dv", _np(dv), rv, tol, row_rms=True)
     assert_close("d_rel", _np(dr)[:first_anc], rr[:first_anc], tol, row_rms=True)
     # atomics-free, fixed order: a second run gives the same bits
-    dq2, dk2, dv2, dr2 = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"])
-    out2, lse2 = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale)
+    dq2, dk2, dv2, dr2 = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"], workspace=ws, path=path)
+    out2, lse2 = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, path=path)
     torch.cuda.synchronize()
     for a, b in ((dq, dq2), (dk, dk2), (dv, dv2), (dr, dr2), (out, out2), (lse, lse2)):
         assert torch.equal(a, b)
@@ -141,6 +149,17 @@ def test_config5_sweep_points(n, k):
     c = synth.sweep_configs()["cfg5_n%d_k%d" % (n, k)]
     # the oracle covers two batch entries' worth of work per point; the library runs that same problem
     run_case(c["n"], c["k"], c["flags"], min(c["B"], 2), c["H"], c["d"], c["bf16"], c["seed"], c["std_qkv"], True)
+
+
+@pytest.mark.parametrize("n,k,H,frac", [(16384, 64, 4, None), (65536, 64, 2, 0.5), (65536, 64, 2, None)])
+def test_config5_sweep_points_k64(n, k, H, frac):
+    """The k = 64 column of the sweep at its two long sequence lengths: one batch entry and a reduced number of
+    heads keep the fp64 oracle to about a minute; batch entries and heads are independent problems on the same
+    graph.  With half of the planned workspace the warp-level backward takes its pairs in more than one pass."""
+    from paper_1911_04070_b200 import binding, synth
+    c = synth.sweep_configs()["cfg5_n%d_k%d" % (n, k)]
+    run_case(c["n"], c["k"], c["flags"], 1, H, c["d"], c["bf16"], c["seed"], c["std_qkv"], True,
+             path=binding.BPT_PATH_MMA if frac is not None else 0, bwd_workspace_frac=frac)
 
 
 def test_argument_errors_do_not_launch():

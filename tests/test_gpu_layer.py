@@ -67,6 +67,45 @@ def test_fp32_left_only_with_lengths_root_readout():
     _run(n=32, k=3, left_only=True, D=64, H=2, F=64, n_layers=1, dtype=torch.float32, lengths=[32, 19], readout="root", tol=2e-4)
 
 
-def test_bf16_layer_tiled_kernels():
+def test_bf16_layer_tiled_kernels(monkeypatch):
+    """The layer in bf16 runs the tiled kernels with lengths.  What those kernels produce inside the layer is
+    compared element by element: the attention's inputs and output are recorded on the way through the layer
+    and the oracle is evaluated on exactly those inputs.  The layer's own output and parameter gradients also pass
+    through PyTorch's bf16 linear / norm / relu operators and are held to a 2-norm bound only."""
     import torch
+    from oracle import ctwin
+    from paper_1911_04070_b200 import binding, layer
+    from parity import TOL, assert_close
+    seen = []
+    real_fwd, real_bwd = binding.bpt_attn_fwd, binding.bpt_attn_bwd
+
+    def rec_fwd(g, q, k, v, rel_emb, scale, **kw):
+        out, lse = real_fwd(g, q, k, v, rel_emb, scale, **kw)
+        seen.append(dict(kind="fwd", g=g, q=q, k=k, v=v, r=rel_emb, scale=scale, lengths=kw.get("lengths"), out=out, lse=lse))
+        return out, lse
+
+    def rec_bwd(g, q, k, v, rel_emb, scale, out, lse, d_out, **kw):
+        grads = real_bwd(g, q, k, v, rel_emb, scale, out, lse, d_out, **kw)
+        seen.append(dict(kind="bwd", g=g, q=q, k=k, v=v, r=rel_emb, scale=scale, lengths=kw.get("lengths"), out=out,
+                         d_out=d_out, grads=grads))
+        return grads
+
+    monkeypatch.setattr(binding, "bpt_attn_fwd", rec_fwd)
+    monkeypatch.setattr(binding, "bpt_attn_bwd", rec_bwd)
     _run(n=128, k=4, left_only=False, D=128, H=2, F=128, n_layers=1, dtype=torch.bfloat16, lengths=[128, 77], readout="tokens", tol=1e-1)
+    assert [s["kind"] for s in seen] == ["fwd", "bwd"]
+    f64 = lambda t: t.detach().float().cpu().numpy().astype(np.float64)
+    for s in seen:
+        ref = ctwin.CGraph(s["g"].n, s["g"].k, 0)
+        lens = s["lengths"].cpu().numpy()
+        q, k, v, r = (f64(s[a]) for a in ("q", "k", "v", "r"))
+        if s["kind"] == "fwd":
+            o_ref, lse_ref = ctwin.attn_fwd_varlen(ref, q, k, v, r, s["scale"], lens)
+            assert_close("attention out inside the layer", f64(s["out"]), o_ref, TOL["bf16"])
+            assert_close("attention lse inside the layer", f64(s["lse"]), lse_ref, TOL["bf16"])
+        else:
+            want = ctwin.attn_bwd_varlen(ref, q, k, v, r, s["scale"], f64(s["d_out"]), lens, out=f64(s["out"]))
+            fa = 1 + 2 * ref.L * (s["g"].k + 1)
+            for name, a, b in zip(("dq", "dk", "dv"), s["grads"][:3], want[:3]):
+                assert_close("attention %s inside the layer" % name, f64(a), b, TOL["bf16"], row_rms=True)
+            assert_close("attention d_rel inside the layer", f64(s["grads"][3])[:fa], want[3][:fa], TOL["bf16"], row_rms=True)

@@ -1,62 +1,60 @@
-"""The tiled backward works through the (batch entry, head) pairs in passes when its partial rows would
-exceed the per-pass cap, adding d_rel up over the passes.  With the cap lowered through the
-environment (read once per process, hence the child process) a mid-sized problem takes many passes and
-must still match the oracle and the single-pass result bit for bit."""
-import os
-import subprocess
-import sys
-
+"""The tiled backward works through the (batch entry, head) pairs in passes when the workspace it is
+given holds the partial rows of only some of them, adding d_rel up over the passes.  With a workspace
+a sixth of the planned size a mid-sized problem takes several passes and must still match the oracle,
+and the single-pass result bit for bit."""
+import numpy as np
 import pytest
+
+from parity import TOL, assert_close
 
 pytestmark = pytest.mark.gpu
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
-CHILD = r"""
-import sys
-sys.path.insert(0, %(root)r); sys.path.insert(0, %(tests)r)
-import numpy as np, torch
-from oracle import ctwin
-from paper_1911_04070_b200 import binding, synth
-from parity import TOL, assert_close
-n, k, flags, B, H, d = 1024, 16, 0, 3, 5, 64
-ref = ctwin.CGraph(n, k, flags)
-x = synth.make_inputs(B, ref.n_nodes, H, d, ref.n_rel, seed=21, std_qkv=0.5, std_rel=0.3, bf16=True)
-t = {a: torch.from_numpy(b).to("cuda:0", torch.bfloat16) for a, b in x.items()}
-g = binding.bpt_build_graph(n, k, flags, device="cuda:0")
-need = binding.bpt_attn_workspace_bytes(g, B, H, d, binding.BPT_BF16, True)
-out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125)
-binding.bpt_trace_begin(400)
-grads = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125, out, lse, t["d_out"])
-passes = sum(1 for a, _ in binding.bpt_trace_end(400) if a == "bwd_tile")
-torch.cuda.synchronize()
-o64 = out.float().cpu().numpy().astype(np.float64)
-want = ctwin.attn_bwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], 0.125, x["d_out"], out=o64)
-fa = 1 + 2 * ref.L * (k + 1)
-for name, a, b in zip(("dq", "dk", "dv"), grads[:3], want[:3]):
-    assert_close(name, a.float().cpu().numpy(), b, TOL["bf16"], row_rms=True)
-assert_close("d_rel", grads[3].cpu().numpy()[:fa], want[3][:fa], TOL["bf16"], row_rms=True)
-torch.save([a.cpu() for a in grads], %(dump)r)
-print("passes", passes, "workspace", need)
-"""
-
-
-def _run(env_extra, dump):
-    env = dict(os.environ, **env_extra)
-    code = CHILD % {"root": ROOT, "tests": os.path.join(ROOT, "tests"), "dump": dump}
-    res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=900)
-    assert res.returncode == 0, res.stdout[-2000:] + res.stderr[-4000:]
-    words = res.stdout.split()
-    return int(words[words.index("passes") + 1]), int(words[words.index("workspace") + 1])
-
-
-def test_many_passes_match_one_pass(tmp_path):
+def _backward(g, t, out, lse, ws_bytes):
     import torch
-    one, ws_one = _run({}, str(tmp_path / "one.pt"))
-    many, ws_many = _run({"BPT_BWD_PASS_MB": "24"}, str(tmp_path / "many.pt"))
-    assert one == 1 and many >= 4 and ws_many < ws_one
-    a, b = torch.load(tmp_path / "one.pt"), torch.load(tmp_path / "many.pt")
-    for name, x, y in zip(("dq", "dk", "dv"), a[:3], b[:3]):
-        assert torch.equal(x, y), name           # per-pair work does not depend on the pass it runs in
-    # d_rel is summed pass by pass (another, still fixed, order): equal up to fp32 rounding
-    assert torch.allclose(a[3], b[3], rtol=1e-4, atol=1e-6 * float(a[3].abs().max()))
+    from paper_1911_04070_b200 import binding
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda:0")
+    binding.bpt_trace_begin(400)
+    grads = binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125, out, lse, t["d_out"], workspace=ws,
+                                 path=binding.BPT_PATH_MMA)
+    passes = sum(1 for a, _ in binding.bpt_trace_end(400) if a == "bwd_tile")
+    assert binding.bpt_check(ws) == 0
+    return grads, passes
+
+
+def test_many_passes_match_one_pass():
+    import torch
+    from oracle import ctwin
+    from paper_1911_04070_b200 import binding, synth
+    n, k, flags, B, H, d = 1024, 16, 0, 3, 5, 64
+    ref = ctwin.CGraph(n, k, flags)
+    x = synth.make_inputs(B, ref.n_nodes, H, d, ref.n_rel, seed=21, std_qkv=0.5, std_rel=0.3, bf16=True)
+    t = {a: torch.from_numpy(b).to("cuda:0", torch.bfloat16) for a, b in x.items()}
+    g = binding.bpt_build_graph(n, k, flags, device="cuda:0")
+    ws_one = binding.bpt_attn_workspace_bytes(g, B, H, d, binding.BPT_BF16, True)
+    ws_min = binding.bpt_attn_bwd_min_workspace_bytes(g, B, H, d, binding.BPT_BF16)
+    ws_many = max(ws_one // 6, ws_min)
+    assert ws_min <= ws_many < ws_one
+    out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125)
+    one, passes_one = _backward(g, t, out, lse, ws_one)
+    many, passes_many = _backward(g, t, out, lse, ws_many)
+    least, passes_least = _backward(g, t, out, lse, ws_min)
+    assert passes_one == 1 and 1 < passes_many < passes_least == B * H
+
+    o64 = out.float().cpu().numpy().astype(np.float64)
+    want = ctwin.attn_bwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], 0.125, x["d_out"], out=o64)
+    fa = 1 + 2 * ref.L * (k + 1)
+    for grads in (many, least):
+        for name, a, b in zip(("dq", "dk", "dv"), grads[:3], want[:3]):
+            assert_close(name, a.float().cpu().numpy(), b, TOL["bf16"], row_rms=True)
+        assert_close("d_rel", grads[3].cpu().numpy()[:fa], want[3][:fa], TOL["bf16"], row_rms=True)
+        for name, x1, y1 in zip(("dq", "dk", "dv"), one[:3], grads[:3]):
+            assert torch.equal(x1, y1), name       # per-pair work does not depend on the pass it runs in
+        # d_rel is summed pass by pass (another, still fixed, order): equal up to fp32 rounding
+        assert torch.allclose(one[3], grads[3], rtol=1e-4, atol=1e-6 * float(one[3].abs().max()))
+
+    # a workspace below the minimum is refused on the host
+    with pytest.raises(binding.BptError) as ei:
+        binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125, out, lse, t["d_out"],
+                             workspace=torch.empty(ws_min - 256, dtype=torch.uint8, device="cuda:0"), path=binding.BPT_PATH_MMA)
+    assert ei.value.status == 3
