@@ -690,22 +690,89 @@ size_t pairs_for_budget(const TreeParams& t, const ChunkPlan& plan, int B, int H
 
 }  // namespace
 
+// ---- tensor-memory path (attn_bwd_q_tc5.cu, attn_bwd_kv_tc5.cu): no partial rows; its workspace holds the row
+// terms of all pairs and, per pass, the span pass's blocks and the d_rel partials ----
+bool bwd_q_tc5_fits(const TreeParams& t);
+bpt_status launch_bwd_q_tc5(const AttnProblem& p, float* delta);
+size_t bwd_kv_tc5_drel_floats(const TreeParams& t, int n_pairs);
+bpt_status launch_bwd_kv_tc5(const AttnProblem& p, int pair0, int n_pairs, const float* delta, const float* aff_slab, float* drel_part);
+
+namespace {
+
+struct Tc5Workspace {
+    float *delta, *aff_slab, *ext_dq, *drel_part;
+    int pairs_per_pass;
+    size_t bytes;
+};
+
+Tc5Workspace carve_tc5(const TreeParams& t, int B, int H, size_t pairs, void* base) {
+    Tc5Workspace w;
+    w.pairs_per_pass = (int)pairs;
+    char* c = (char*)base;
+    size_t off = 0;
+    w.delta = (float*)(c + off); off += align256(sizeof(float) * (size_t)B * H * t.n);
+    w.aff_slab = (float*)(c + off); off += align256(sizeof(float) * bwd_span_slab_floats(t, (int)pairs));
+    w.ext_dq = (float*)(c + off); off += align256(sizeof(float) * bwd_span_ext_floats(t, (int)pairs));
+    w.drel_part = (float*)(c + off); off += align256(sizeof(float) * bwd_kv_tc5_drel_floats(t, (int)pairs));
+    w.bytes = off;
+    return w;
+}
+
+size_t tc5_pairs_for_budget(const TreeParams& t, int B, int H, size_t budget) {
+    const size_t all = (size_t)B * H;
+    const size_t fixed = carve_tc5(t, B, H, 0, nullptr).bytes, per_pair = carve_tc5(t, B, H, 1, nullptr).bytes - fixed;
+    size_t pairs = budget > fixed ? (budget - fixed) / per_pair : 0;
+    if (pairs > all) pairs = all;
+    while (pairs < all && carve_tc5(t, B, H, pairs + 1, nullptr).bytes <= budget) ++pairs;
+    return pairs < 1 ? 1 : pairs;
+}
+
+// The tensor-memory kernels take whole tiles of 128 tokens and pay for their hand-offs where a level holds
+// enough nodes per token; bpt_attn_options.path forces either family.
+bool want_bwd_tc5(const TreeParams& t, uint32_t path) {
+    if (path == BPT_PATH_MMA || !bwd_q_tc5_fits(t)) return false;
+    return path == BPT_PATH_TC5 || t.k >= 32;
+}
+
+bpt_status launch_bwd_tc5(const AttnProblem& p) {
+    const TreeParams& t = p.tree;
+    const Tc5Workspace ws = carve_tc5(t, p.B, p.H, tc5_pairs_for_budget(t, p.B, p.H, p.workspace_bytes), p.workspace);
+    if (ws.bytes > p.workspace_bytes) return BPT_ERR_WORKSPACE;
+    bpt_status s = launch_bwd_q_tc5(p, ws.delta);  // token dq and the row terms of every pair
+    const int total = p.B * p.H;
+    for (int pair0 = 0; pair0 < total && s == BPT_OK; pair0 += ws.pairs_per_pass) {
+        const int np = min(ws.pairs_per_pass, total - pair0);
+        s = launch_bwd_span(p, pair0, np, ws.ext_dq, ws.aff_slab);  // span dq; per token the affiliated edges' share of dk / dv
+        if (s == BPT_OK) s = launch_bwd_kv_tc5(p, pair0, np, ws.delta, ws.aff_slab, ws.drel_part);
+    }
+    return s;
+}
+
+}  // namespace
+
 bool bwd_tile_eligible(const bpt_graph& g, int d, bpt_dtype dtype) {
     return tile_path(g.dims.n, g.dims.k, d, dtype == BPT_BF16);
 }
 
 // minimal: the smallest workspace the backward runs with (one pair per pass); otherwise the planned size.
+// Either kernel family may be asked for through the options, so the sizes cover both.
 size_t bwd_tile_workspace_bytes(const bpt_graph& g, int B, int H, bool minimal) {
     TreeParams t;
     tree_params_from_dims(g.dims, &t);
     const ChunkPlan plan = make_plan(t);
     const size_t pairs = minimal ? 1 : pairs_for_budget(t, plan, B, H, kPassBytes);
-    return carve_tile(t, plan, pairs, nullptr).bytes;
+    size_t bytes = carve_tile(t, plan, pairs, nullptr).bytes;
+    if (bwd_q_tc5_fits(t)) {
+        const size_t tp = minimal ? 1 : tc5_pairs_for_budget(t, B, H, kPassBytes);
+        bytes = max(bytes, carve_tc5(t, B, H, tp, nullptr).bytes);
+    }
+    return bytes;
 }
 
 
 bpt_status launch_bwd_tile(const AttnProblem& p) {
     const TreeParams& t = p.tree;
+    if (want_bwd_tc5(t, p.path)) return launch_bwd_tc5(p);
     const ChunkPlan plan = make_plan(t);
     const int chunks = plan.n_left + plan.n_right, tiles = t.n / (kTileTokens * plan.group), N = 2 * t.n - 1;  // tiles: groups
     const TileWorkspace ws = carve_tile(t, plan, pairs_for_budget(t, plan, p.B, p.H, p.workspace_bytes), p.workspace);

@@ -27,10 +27,9 @@
 // (single buffers) and the next V rows into the other of two buffers; O_chunk is collected just
 // before the next chunk's P is written.  Every mbarrier wait gives up after about a second and the
 // kernel then winds down.
-#include <cuda.h>
-
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
+#include "tc5_host.cuh"
 #include "tc5_tools.cuh"
 #include "tile_geom.cuh"
 
@@ -434,49 +433,9 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right,
 
 }  // namespace
 
-namespace {
-
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// The driver's tensor-map encoder, looked up through the runtime (the library does not link libcuda).
-EncodeTiledFn encode_tiled() {
-    static EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) != cudaSuccess ||
-            qr != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// Map over a [B, N, H, 64] bf16 tensor: a box is 16 consecutive nodes of one (batch entry, head), 128-byte swizzle.
-bool node_rows_map(CUtensorMap* m, const void* base, int B, int N, int H) {
-    const cuuint64_t dims[4] = {64, (cuuint64_t)H, (cuuint64_t)N, (cuuint64_t)B};
-    const cuuint64_t strides[3] = {128, (cuuint64_t)H * 128, (cuuint64_t)N * H * 128};
-    const cuuint32_t box[4] = {64, 1, 16, 1}, estr[4] = {1, 1, 1, 1};
-    return encode_tiled()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-// Map over the [n_rel, 64] relation table: a box is 16 consecutive relations.
-bool rel_rows_map(CUtensorMap* m, const void* base, int n_rel) {
-    const cuuint64_t dims[2] = {64, (cuuint64_t)n_rel};
-    const cuuint64_t strides[1] = {128};
-    const cuuint32_t box[2] = {64, 16}, estr[2] = {1, 1};
-    return encode_tiled()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-}  // namespace
-
 // The tensor-memory kernel takes whole tiles of 128 tokens.
 bool fwd_tc5_eligible(const AttnProblem& p) {
-    if (!encode_tiled()) return false;
+    if (!tc5::encode_tiled()) return false;
     if (!tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16) || p.tree.n < kTcTokens) return false;
     int n_left, n_right;
     context_levels(p.tree, &n_left, &n_right);
@@ -494,8 +453,8 @@ bpt_status launch_fwd_tc5(const AttnProblem& p, int* status) {
         return BPT_ERR_CUDA;
     alignas(64) CUtensorMap tm_k, tm_v, tm_r;
     const int N = 2 * p.tree.n - 1;
-    if (!encode_tiled() || !node_rows_map(&tm_k, p.k, p.B, N, p.H) || !node_rows_map(&tm_v, p.v, p.B, N, p.H) ||
-        !rel_rows_map(&tm_r, p.rel_emb, p.g->dims.n_rel))
+    if (!tc5::encode_tiled() || !tc5::node_rows_map(&tm_k, p.k, p.B, N, p.H) || !tc5::node_rows_map(&tm_v, p.v, p.B, N, p.H) ||
+        !tc5::rel_rows_map(&tm_r, p.rel_emb, p.g->dims.n_rel))
         return BPT_ERR_CUDA;
     const dim3 grid(p.tree.n / kTcTokens, p.H, p.B);
     kernel<<<grid, kTcThreads, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q,

@@ -46,8 +46,8 @@ def test_many_passes_match_one_pass():
     fa = 1 + 2 * ref.L * (k + 1)
     for grads in (many, least):
         for name, a, b in zip(("dq", "dk", "dv"), grads[:3], want[:3]):
-            assert_close(name, a.float().cpu().numpy(), b, TOL["bf16"], row_rms=True)
-        assert_close("d_rel", grads[3].cpu().numpy()[:fa], want[3][:fa], TOL["bf16"], row_rms=True)
+            assert_close(name, a.float().cpu().numpy(), b, TOL["bf16"], row_rms=(name == "dq"))
+        assert_close("d_rel", grads[3].cpu().numpy()[:fa], want[3][:fa], TOL["bf16"])
         for name, x1, y1 in zip(("dq", "dk", "dv"), one[:3], grads[:3]):
             assert torch.equal(x1, y1), name       # per-pair work does not depend on the pass it runs in
         # d_rel is summed pass by pass (another, still fixed, order): equal up to fp32 rounding
