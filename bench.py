@@ -43,20 +43,44 @@ KERNEL_MODEL = {
     "fwd_rows": (("fwd",), "all"), "bwd_dst": (("bwd_dst",), "all"), "bwd_src": (("bwd_src",), "all"),
     "fwd_tile": (("fwd",), "token"), "fwd_tc5": (("fwd",), "token"), "fwd_span": (("fwd",), "span"),
     "bwd_tile": (("bwd_dst", "bwd_src"), "token"), "bwd_span": (("bwd_dst", "bwd_src"), "span"),
+    "bwd_q_tc5": (("bwd_dst",), "token"), "bwd_kv_tc5": (("bwd_src",), "token"),
 }
-# DRAM bytes (read + write) per (batch entry, head) pair of one launch, from the ncu captures summarised
-# under profiles/ (taken at batch 1; every pair is an independent problem, so traffic scales with pairs).
-# An entry is dropped (traffic = null) when its kernel changes after the capture.
-NCU_DRAM_BYTES_PER_PAIR = {"fwd_tc5": 41.28e6 / 8, "bwd_tile": 380.1e6 / 8}  # profiles/tile_kernels_full_cfg4_batch1.md
+# DRAM bytes (read + write) per (batch entry, head) pair of one launch, from ncu captures of the character-LM
+# shape at batch 1 (n = 8192, k = 64, left-only, 8 heads; every pair is an independent problem, so traffic
+# scales with pairs).  Each figure is tied to the source file of its kernel by a hash taken when the counters
+# were read; when the file has changed since, the bench reports traffic = null instead of a stale number.
+NCU_DRAM_BYTES_PER_PAIR = {
+    # kernel: (bytes per pair, source file, sha256 of the file at capture time (first 16 hex digits))
+    "fwd_tc5": (41.28e6 / 8, "attn_fwd_tc5.cu", ""),
+    "bwd_q_tc5": (61.13e6 / 8, "attn_bwd_q_tc5.cu", ""),
+    "bwd_kv_tc5": (106.98e6 / 8, "attn_bwd_kv_tc5.cu", ""),
+}
+FLOPS_PER_EDGE_HEAD = {"fwd": 6, "bwd": 14}   # x d_head: q.k, q.r, P.v forward; s again, dP, dq, dk, dv, d_rel backward
+
+
+def ncu_traffic_per_pair(kernel):
+    """ncu DRAM bytes per pair for `kernel`, or None when unknown or taken from an older version of its source."""
+    import hashlib
+    ent = NCU_DRAM_BYTES_PER_PAIR.get(kernel)
+    if ent is None:
+        return None
+    per_pair, fname, digest = ent
+    path = os.path.join(ROOT, "paper_1911_04070_b200", "csrc", fname)
+    try:
+        now = hashlib.sha256(open(path, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    return per_pair if digest and now == digest else None
 
 
 def load_peaks():
+    """(HBM GB/s, sustained bf16 TFLOP/s, "measured" | "fallback")."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return float(p["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(p["hbm_gbs"]), float(p.get("bf16_tflops_sustained", 1400.0)), "measured"
+    return 6650.0, 1400.0, "fallback"
 
 
 def all_configs():
@@ -356,8 +380,9 @@ def run_ours(args, cfg_name, cfg):
     for name, ms in marks:
         per.setdefault(name, []).append(ms)
     total_ms = max(sum(m for _, m in marks), 1e-9)
-    kernels = {name: {"launches": len(v), "avg_ms": sum(v) / len(v), "share": sum(v) / total_ms} for name, v in per.items()}
-    peak, peak_kind = load_peaks()
+    kernels = {name: {"launches": len(v), "avg_ms": sum(v) / len(v), "min_ms": min(v), "median_ms": statistics.median(v),
+                      "max_ms": max(v), "share": sum(v) / total_ms} for name, v in per.items()}
+    peak, tf_peak, peak_kind = load_peaks()
     E_span = cfg["n"] * (cfg["n"].bit_length() - 1)          # affiliated edges: one per token and level
     edges_of = {"all": E, "token": E - E_span, "span": E_span}
     modelled = [a for a in kernels if a in KERNEL_MODEL]
@@ -367,12 +392,12 @@ def run_ours(args, cfg_name, cfg):
         passes, rows = KERNEL_MODEL[dominant]
         alg_bytes = sum(GATHER_BYTES_PER_EDGE_HEAD[a](d, esize) for a in passes) * B * H * edges_of[rows]
         achieved = alg_bytes / (kernels[dominant]["avg_ms"] * 1e-3) / 1e9
-        per_pair = NCU_DRAM_BYTES_PER_PAIR.get(dominant)
+        per_pair = ncu_traffic_per_pair(dominant)
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " copy bandwidth",
                     "unit": "GB/s", "frac": achieved / peak, "traffic": None if per_pair is None else per_pair * B * H,
                     "algorithmic_bytes": alg_bytes,
                     "model": "gather model: K/V (and, backward, Q/dO) rows fetched per edge and head with no on-chip reuse "
-                             "credited; the tiled kernels stage each level's node range once per 64 tokens, so frac > 1 "
+                             "credited; the tiled kernels stage each level's node range once per tile, so frac > 1 "
                              "measures that reuse, and `traffic` (ncu DRAM bytes) shows what HBM really moved"}
     # whole-step fraction of the gather-model roofline (the target figure of the benchmark definition)
     gathered = sum(GATHER_BYTES_PER_EDGE_HEAD[a](d, esize) for a in (["fwd", "bwd_dst", "bwd_src"] if do_bwd else ["fwd"])) * B * H * E
@@ -380,7 +405,24 @@ def run_ours(args, cfg_name, cfg):
     # lower bound of a step: every input and output tensor crosses HBM once
     compulsory = ((4 + (5 if do_bwd else 0)) * B * N * H * d * esize + 4 * B * N * H * (2 if do_bwd else 1))
     compulsory_ms = compulsory / (peak * 1e9) * 1e3
+    # true lower bound: the slower of the compulsory HBM traffic and the algorithmic FLOPs on the tensor cores
+    flops_alg = (FLOPS_PER_EDGE_HEAD["fwd"] + (FLOPS_PER_EDGE_HEAD["bwd"] if do_bwd else 0)) * d * B * H * E
+    flops_ms = flops_alg / (tf_peak * 1e12) * 1e3
+    lower_bound_ms = max(compulsory_ms, flops_ms)
+    if roofline:   # the same bound for the dominant kernel alone: its share of the algorithmic FLOPs, its own compulsory tensors
+        passes, rows = KERNEL_MODEL[dominant]
+        k_flops = sum({"fwd": 6, "bwd_dst": 8, "bwd_src": 6}[a] for a in passes) * d * B * H * edges_of[rows]
+        k_tensors = {"fwd": 4, "bwd_dst": 6, "bwd_src": 6}   # node-major tensors the pass must read or write once
+        k_bytes = sum(k_tensors[a] for a in passes) * B * N * H * d * esize
+        k_lb = max(k_bytes / (peak * 1e9), k_flops / (tf_peak * 1e12)) * 1e3
+        roofline.update(lower_bound_ms=k_lb, lower_bound_frac=k_lb / kernels[dominant]["avg_ms"],
+                        flops_alg=k_flops, compulsory_bytes=k_bytes)
 
+    # per-step series from the per-launch marks (launch order repeats every step)
+    per_step = []
+    if marks and len(marks) % args.steps == 0:
+        n_per = len(marks) // args.steps
+        per_step = [sum(m for _, m in marks[i * n_per:(i + 1) * n_per]) for i in range(args.steps)]
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -392,11 +434,15 @@ def run_ours(args, cfg_name, cfg):
         "edge_heads_per_s": value * H, "tokens_per_s": world * B * cfg["n"] / (ms_step * 1e-3),
         "hbm_roofline_frac_step": step_roof_ms / ms_step, "hbm_roofline_ms_step": step_roof_ms,
         "compulsory_hbm_ms_step": compulsory_ms, "compulsory_hbm_frac_step": compulsory_ms / ms_step,
+        "flops_alg": flops_alg, "flops_ms_at_sustained_bf16_peak": flops_ms, "tensor_peak_tflops": tf_peak,
+        "lower_bound_ms": lower_bound_ms, "lower_bound_frac": lower_bound_ms / ms_step,
         "clocks": clocks,
         "e2e": {"value": world * B * E / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "overlap": "copies of the neighbouring steps run under the kernels (three streams, two buffer sets)"},
         "gpu_launches": len(marks),
+        "step_ms_series": {"min": min(per_step), "median": statistics.median(per_step), "max": max(per_step),
+                           "first": per_step[0], "last": per_step[-1]} if per_step else None,
         "kernels": kernels,
         "roofline": roofline,
     }
@@ -529,6 +575,11 @@ def main():
         cfg["B"] = args.batch
     if args.impl == "reference":
         run_reference(args, args.config, cfg)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # asked for N GPUs without a launcher: start one rank per GPU of this node and let them run this script
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(29500 + os.getpid() % 2000), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd, env=dict(os.environ, NCCL_DEBUG=os.environ.get("NCCL_DEBUG", "INFO"))))
     else:
         if args.warmup < 3:
             args.warmup = 3

@@ -37,7 +37,7 @@ constexpr int kKvKeys = 128;                     // nodes per CTA
 constexpr int kKvQB = 64;                        // query tokens per item
 constexpr int kKvTpr = 4;                        // threads per key row
 constexpr int kKvRowThreads = kKvKeys * kKvTpr;  // 16 warps
-constexpr int kKvThreads = kKvRowThreads + 64;   // + load warp + MMA warp
+constexpr int kKvThreads = kKvRowThreads + 96;   // + load warp + two MMA warps
 constexpr int kKvCols = kKvQB / kKvTpr;          // query columns per thread and item
 constexpr int kKvRing = 3;
 constexpr int kKvRelRows = 80;                   // relation rows per side (k + 2 <= 66), in 16-row boxes
@@ -116,6 +116,49 @@ __device__ __forceinline__ void tile_of(int n, int L, int x, int* level, int* m0
     *level = 0; *m0 = 0;
 }
 
+// One item's share of a row thread: its key node m against kKvCols query columns.  Predicated, no branch per element.
+// kSide: 1 = the keys are right context of the queries (offset m - lo), 0 = left context (offset hi - m).
+// Two phases, so that no shared-memory store stands between the loads of different elements (the compiler must
+// assume the by-offset stores alias the tables): first every weight, then every store.  The by-offset store of a
+// missing edge goes, with value zero, to row 127 of the tile, which is no relation offset.
+template <int kSide, bool kDrop>
+__device__ __forceinline__ void kv_rows_item(const uint32_t (&sv)[kKvCols], const uint32_t (&dv)[kKvCols], const QMeta* __restrict__ mq,
+                                             const float* __restrict__ bias_col, unsigned char* __restrict__ skw, int m, int part,
+                                             float scale_log2e, const DropoutParams& drop, uint32_t pair, uint32_t dst0, uint32_t src,
+                                             uint32_t (&pp)[kKvCols / 2], uint32_t (&dd)[kKvCols / 2]) {
+    uint32_t at[kKvCols];  // byte offset of each element's by-offset store
+#pragma unroll
+    for (int x = 0; x < kKvCols; x += 2) {
+        float pv[2], dsv[2];
+#pragma unroll
+        for (int y = 0; y < 2; ++y) {
+            const QMeta a = mq[x + y];
+            const bool in = m >= a.lo && m <= a.hi;
+            const int off = kSide ? m - a.lo : a.hi - m;
+            const int col = part * kKvCols + x + y;
+            const float bias = in ? bias_col[(x + y) * kKvBiasStride + off] : 0.f;
+            float pr = ex2f(fmaf(__uint_as_float(sv[x + y]), scale_log2e, bias));
+            float dp = __uint_as_float(dv[x + y]), d;
+            if constexpr (kDrop) {  // dP = W d_out.v, the weight that reaches dv is W P, dS keeps the undropped P
+                const float wgt = dropout_weight(drop, pair, dst0 + (uint32_t)(x + y), src);
+                d = pr * (dp * wgt - a.delta);
+                pr *= wgt;
+            } else {
+                d = pr * (dp - a.delta);
+            }
+            pv[y] = in ? pr : 0.f;
+            dsv[y] = in ? d : 0.f;
+            const int so = in ? off : kKvKeys - 1;
+            at[x + y] = (uint32_t)(so * 128 + ((((col >> 3) ^ so) & 7) << 4) + (col & 7) * 2);
+        }
+        pp[x >> 1] = pack_bf16(pv[0], pv[1]);
+        dd[x >> 1] = pack_bf16(dsv[0], dsv[1]);
+    }
+#pragma unroll
+    for (int x = 0; x < kKvCols; ++x)
+        *reinterpret_cast<uint16_t*>(skw + at[x]) = (uint16_t)((x & 1) ? dd[x >> 1] >> 16 : dd[x >> 1] & 0xffffu);
+}
+
 template <bool kDrop>
 __global__ void __launch_bounds__(kKvThreads, 1)
 bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
@@ -153,7 +196,7 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
     auto bar = [&](int i) { return bar_u + 8u * (uint32_t)i; };
     auto wait = [&](int i, uint32_t parity) {
         if (*abort_s) return;
-        if (!tc5::mbar_wait(bar(i), parity)) *abort_s = 1;
+        if (!tc5::mbar_wait_fast(bar(i), parity)) *abort_s = 1;
     };
     const int len = seq_len(lengths, b, t.n);
     const bool side_on[2] = {level < n_left, level < n_right};
@@ -226,8 +269,16 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
                         tc5::tma_load_4d(g_u + rb * (kKvQB * 128) + x * 2048, &tm_g, 0, h, q0 + 16 * x, b, bar(kvQFull + rb));
                     }
                 }
+                // per query: node range at this level, lse and row term (the two loads fly while the ranges are walked)
+                float lv[kKvQB / 32], dl[kKvQB / 32];
 #pragma unroll
-                for (int x = 0; x < kKvQB / 32; ++x) {  // per query: node range at this level, lse and row term
+                for (int x = 0; x < kKvQB / 32; ++x) {
+                    const int i = q0 + lane + 32 * x;
+                    lv[x] = __ldg(lse + ((size_t)b * N_nodes + i) * H + h);
+                    dl[x] = __ldg(delta_in + (size_t)pair * t.n + i);
+                }
+#pragma unroll
+                for (int x = 0; x < kKvQB / 32; ++x) {
                     const int i = q0 + lane + 32 * x;
                     int2 rg = level_range(t, i, side, level);
                     if (len < t.n) {  // short sequence: a placeholder token attends nothing, right ranges end at the last real node
@@ -236,64 +287,64 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
                     }
                     QMeta qm;
                     qm.lo = rg.x; qm.hi = rg.y;
-                    qm.lse2 = lse[((size_t)b * N_nodes + i) * H + h] * kLog2e;
-                    qm.delta = delta_in[(size_t)pair * t.n + i];
+                    qm.lse2 = lv[x] * kLog2e;
+                    qm.delta = dl[x];
                     meta_s[rb * kKvQB + lane + 32 * x] = qm;
                 }
                 tc5::mbar_arrive(bar(kvQFull + rb));
             }
         }
     } else if (w == kKvRowThreads / 32 + 1) {
-        // =============== MMA warp: one thread issues every tensor-core instruction ===============
+        // =============== first MMA warp: one thread issues S^T, dP^T and QR^T of every item ===============
         if (lane == 0 && J > 0) {
-            const uint32_t id_t = tc5::instr_desc(kKvKeys, kKvQB, 0, 0), id_o = tc5::instr_desc(kKvKeys, 64, 0, 1);
-            auto issue_a = [&](int j) {  // S^T, dP^T and QR^T of item j
+            const uint32_t id_t = tc5::instr_desc(kKvKeys, kKvQB, 0, 0);
+            const uint32_t k_lo = tc5::desc_lo_k_major(k_u), v_lo = tc5::desc_lo_k_major(v_u);
+            for (int j = 0; j < J && !*abort_s; ++j) {
                 int side, q0;
                 item_of(j, side, q0);
                 const int rb = j % kKvRing, ru = j / kKvRing;
                 if (j == 0) wait(kvTiles, 0);
                 wait(kvQFull + rb, ru & 1);
                 if (j > 0) wait(kvSFree, (j - 1) & 1);
-                if (*abort_s) return;
+                if (*abort_s) break;
                 tc5::fence_after_sync();
-                const uint32_t qq = q_u + rb * (kKvQB * 128), gg = g_u + rb * (kKvQB * 128), rr = r_u + side * (kKvKeys * 128);
+                const uint32_t q_lo = tc5::desc_lo_k_major(q_u + rb * (kKvQB * 128)), g_lo = tc5::desc_lo_k_major(g_u + rb * (kKvQB * 128)),
+                               r_lo = tc5::desc_lo_k_major(r_u + side * (kKvKeys * 128));
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    tc5::mma(tbase + kKvColS, tc5::desc_k_major(k_u + ks * 32), tc5::desc_k_major(qq + ks * 32), id_t, ks > 0);
+                for (int ks = 0; ks < 4; ++ks) tc5::mma_lo(tbase + kKvColS, k_lo + ks * 2, q_lo + ks * 2, id_t, ks > 0);
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    tc5::mma(tbase + kKvColDP, tc5::desc_k_major(v_u + ks * 32), tc5::desc_k_major(gg + ks * 32), id_t, ks > 0);
+                for (int ks = 0; ks < 4; ++ks) tc5::mma_lo(tbase + kKvColDP, v_lo + ks * 2, g_lo + ks * 2, id_t, ks > 0);
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    tc5::mma(tbase + kKvColQR, tc5::desc_k_major(rr + ks * 32), tc5::desc_k_major(qq + ks * 32), id_t, ks > 0);
+                for (int ks = 0; ks < 4; ++ks) tc5::mma_lo(tbase + kKvColQR, r_lo + ks * 2, q_lo + ks * 2, id_t, ks > 0);
                 tc5::commit(bar(kvSFull));
-            };
-            auto issue_b = [&](int j) {  // dK += dS^T Q_blk, dV += P^T dO_blk, dR_side += skew(dS)^T Q_blk
+            }
+        }
+    } else if (w == kKvRowThreads / 32 + 2) {
+        // =============== second MMA warp: one thread issues dK += dS^T Q_blk, dV += P^T dO_blk, dR_side += skew(dS)^T Q_blk ===============
+        if (lane == 0 && J > 0) {
+            const uint32_t id_o = tc5::instr_desc(kKvKeys, 64, 0, 1);
+            const uint32_t ds_lo = tc5::desc_lo_k_major(ds_u), p_lo = tc5::desc_lo_k_major(p_u);
+            for (int j = 0; j < J && !*abort_s; ++j) {
                 int side, q0;
                 item_of(j, side, q0);
                 const int rb = j % kKvRing;
                 wait(kvDsFull, j & 1);
-                if (*abort_s) return;
+                if (*abort_s) break;
                 tc5::fence_after_sync();
-                const uint32_t qq = q_u + rb * (kKvQB * 128), gg = g_u + rb * (kKvQB * 128);
-                const uint32_t sk = sk_u + (j & 1) * (kKvKeys * 128);
+                const uint32_t q_lo = tc5::desc_lo_mn_major(q_u + rb * (kKvQB * 128)), g_lo = tc5::desc_lo_mn_major(g_u + rb * (kKvQB * 128));
+                const uint32_t sk_lo = tc5::desc_lo_k_major(sk_u + (j & 1) * (kKvKeys * 128));
                 const uint32_t first_all = j > 0, first_side = (side ? j > nb_side[0] : j > 0);
 #pragma unroll
                 for (int kk = 0; kk < kKvQB / 16; ++kk)
-                    tc5::mma(tbase + kKvColDK, tc5::desc_k_major(ds_u + kk * 32), tc5::desc_mn_major(qq + kk * 2048), id_o, (first_all || kk > 0) ? 1u : 0u);
+                    tc5::mma_lo(tbase + kKvColDK, ds_lo + kk * 2, q_lo + kk * (2048 / 16), id_o, (first_all || kk > 0) ? 1u : 0u);
 #pragma unroll
                 for (int kk = 0; kk < kKvQB / 16; ++kk)
-                    tc5::mma(tbase + kKvColDV, tc5::desc_k_major(p_u + kk * 32), tc5::desc_mn_major(gg + kk * 2048), id_o, (first_all || kk > 0) ? 1u : 0u);
+                    tc5::mma_lo(tbase + kKvColDV, p_lo + kk * 2, g_lo + kk * (2048 / 16), id_o, (first_all || kk > 0) ? 1u : 0u);
 #pragma unroll
                 for (int kk = 0; kk < kKvQB / 16; ++kk)
-                    tc5::mma(tbase + kKvColDR + side * 64, tc5::desc_k_major(sk + kk * 32), tc5::desc_mn_major(qq + kk * 2048), id_o, (first_side || kk > 0) ? 1u : 0u);
+                    tc5::mma_lo(tbase + kKvColDR + side * 64, sk_lo + kk * 2, q_lo + kk * (2048 / 16), id_o, (first_side || kk > 0) ? 1u : 0u);
                 tc5::commit(bar(kvQFree + rb));
                 tc5::commit(bar(kvDsFree));
-            };
-            issue_a(0);
-            for (int j = 0; j < J; ++j) {
-                if (j + 1 < J) issue_a(j + 1);
-                issue_b(j);
             }
         }
     } else {
@@ -318,48 +369,29 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
             tc5::tmem_ld_wait();
             tc5::fence_before_sync();
             tc5::mbar_arrive(bar(kvSFree));
-            if (quad < 3 && row < kKvBiasStride) {
+            const QMeta* mq = meta_s + rb * kKvQB + part * kKvCols;
+            if (quad < 3 && row < kKvBiasStride) {  // table entry = scale * log2(e) * q.r - lse * log2(e) of the query
+                float nl[kKvCols];
 #pragma unroll
-                for (int x = 0; x < kKvCols; ++x) bias[(part * kKvCols + x) * kKvBiasStride + row] = __uint_as_float(qr[x]) * scale_log2e;
+                for (int x = 0; x < kKvCols; ++x) nl[x] = -mq[x].lse2;   // all loads before the first store
+#pragma unroll
+                for (int x = 0; x < kKvCols; ++x)
+                    bias[(part * kKvCols + x) * kKvBiasStride + row] = fmaf(__uint_as_float(qr[x]), scale_log2e, nl[x]);
             }
             asm volatile("bar.sync 1, %0;" ::"n"(kKvRowThreads) : "memory");  // the table of this item is complete (and the other by-offset tile is cleared)
             if (j > 0) wait(kvDsFree, (j - 1) & 1);   // the products that read P^T, dS^T of the item before are done
 
             // does any of the warp's 32 keys meet any of this thread group's 16 queries?
-            const QMeta* mq = meta_s + rb * kKvQB + part * kKvCols;
             bool hit = false;
             if (lane < kKvCols) { const QMeta a = mq[lane]; hit = a.lo <= a.hi && a.hi >= mw0 && a.lo <= mw0 + 31; }
             uint32_t pp[kKvCols / 2], dd[kKvCols / 2];
 #pragma unroll
             for (int x = 0; x < kKvCols / 2; ++x) pp[x] = dd[x] = 0u;
             if (__any_sync(0xffffffffu, hit)) {
-#pragma unroll
-                for (int x = 0; x < kKvCols; x += 2) {
-                    float pv[2], dsv[2];
-#pragma unroll
-                    for (int y = 0; y < 2; ++y) {  // branch-free: an edge that does not exist computes on clamped indices and stores zeros
-                        const QMeta a = mq[x + y];
-                        const bool in = m >= a.lo && m <= a.hi;
-                        const int off = in ? (side ? m - a.lo : a.hi - m) : 0;
-                        const int col = part * kKvCols + x + y;
-                        float pr = ex2f(fmaf(__uint_as_float(sv[x + y]), scale_log2e, bias[col * kKvBiasStride + off]) - a.lse2);
-                        float dp = __uint_as_float(dv[x + y]), d;
-                        if constexpr (kDrop) {  // dP = W d_out.v, the weight that reaches dv is W P, dS keeps the undropped P
-                            const float wgt = dropout_weight(drop, (uint32_t)pair, (uint32_t)(q0 + col), (uint32_t)(id0 + m));
-                            d = pr * (dp * wgt - a.delta);
-                            pr *= wgt;
-                        } else {
-                            d = pr * (dp - a.delta);
-                        }
-                        pr = in ? pr : 0.f;
-                        d = in ? d : 0.f;
-                        // row 127 of the by-offset tile is no relation offset: the zeros of missing edges land there
-                        *reinterpret_cast<__nv_bfloat16*>(skw + tile_off(in ? off : kKvKeys - 1, col >> 3) + (col & 7) * 2) = __float2bfloat16_rn(d);
-                        pv[y] = pr; dsv[y] = d;
-                    }
-                    pp[x >> 1] = pack_bf16(pv[0], pv[1]);
-                    dd[x >> 1] = pack_bf16(dsv[0], dsv[1]);
-                }
+                const float* bias_col = bias + part * kKvCols * kKvBiasStride;
+                const uint32_t src = (uint32_t)(id0 + m), dst0 = (uint32_t)(q0 + part * kKvCols);
+                if (side) kv_rows_item<1, kDrop>(sv, dv, mq, bias_col, skw, m, part, scale_log2e, drop, (uint32_t)pair, dst0, src, pp, dd);
+                else kv_rows_item<0, kDrop>(sv, dv, mq, bias_col, skw, m, part, scale_log2e, drop, (uint32_t)pair, dst0, src, pp, dd);
             }
 #pragma unroll
             for (int c = 0; c < kKvCols / 8; ++c) {

@@ -31,7 +31,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kQTok = 128;                      // tokens per CTA
 constexpr int kQTpr = 4;                        // threads per token row
 constexpr int kQRowThreads = kQTok * kQTpr;     // 16 warps
-constexpr int kQThreads = kQRowThreads + 64;    // + load warp + MMA warp
+constexpr int kQThreads = kQRowThreads + 96;    // + load warp + two MMA warps
 constexpr int kQItemCols = 96;                  // key columns per item (three 32-column pieces per warp)
 constexpr int kQPieces = kQItemCols / 32;
 constexpr int kQRelRows = 80;                   // relation rows per chunk (k + 2 <= 66), in 16-row boxes
@@ -53,7 +53,7 @@ struct BwdQSmem {
     static constexpr int row_off = bar_off + 256;                         // lse * log2(e), d_out . out per row
     static constexpr int bnd_off = row_off + 2 * kQTok * 4;               // [chunks][128] short2, [chunks] int2, items
     static size_t bytes(int chunks) {
-        return (size_t)bnd_off + (size_t)chunks * (kQTok * 4 + 8) + (size_t)kQMaxItems * 16 + 16 + 1024;
+        return (size_t)bnd_off + (size_t)chunks * (kQTok * 4 + 8 + 16) + (size_t)kQMaxItems * 16 + 16 + 1024;
     }
 };
 static_assert(BwdQSmem::k_off % 1024 == 0 && BwdQSmem::v_off % 1024 == 0 && BwdQSmem::r_off % 1024 == 0 &&
@@ -77,6 +77,65 @@ __device__ __forceinline__ void quad_bar(int quad) {  // the kQTpr warps that sh
         case 1: asm volatile("bar.sync 2, %0;" ::"n"(32 * kQTpr) : "memory"); break;
         case 2: asm volatile("bar.sync 3, %0;" ::"n"(32 * kQTpr) : "memory"); break;
         default: asm volatile("bar.sync 4, %0;" ::"n"(32 * kQTpr) : "memory"); break;
+    }
+}
+
+constexpr int kQCols = 32 / kQTpr;  // columns of one 32-column piece a thread takes
+
+struct RowCtx {
+    int row, part;
+    float lse, delta, scale_log2e;
+    const float* bias_row;   // bias table entry of offset 0 of this row
+    unsigned char* sk_row;   // this row inside a [128][64] block of the by-offset tile
+    unsigned char* ds_s;
+    uint32_t pair, dst;      // dropout: (batch entry, head) pair and destination node
+};
+
+// One item's share of a row thread: kQCols columns of each of `npieces` 32-column pieces.  kDir = +1: offsets grow
+// with the column (right side), -1: they fall (left side), so that the bias loads and the by-offset stores of
+// consecutive columns are a compile-time stride apart.  Everything is predicated, nothing branches per element.
+template <int kDir, bool kDrop>
+__device__ __forceinline__ void q_rows_item(const RowCtx& rc, const uint32_t (&sv)[kQPieces][kQCols], const uint32_t (&dv)[kQPieces][kQCols],
+                                            int npieces, int ob, int omin, int orange, int ch0, int n_ch,
+                                            const DropoutParams& drop, uint32_t src0) {
+    const int r7 = rc.row & 7;
+    const float* bp = rc.bias_row + ob * kQTok;
+    // Per piece two phases, so that no shared-memory store stands between the table loads of its elements (the
+    // compiler must assume that the tile stores alias the table): first the piece's dS values, then its stores.
+#pragma unroll
+    for (int p = 0; p < kQPieces; ++p) {
+        if (p < npieces) {
+            float dsv[kQCols];
+            uint32_t inm = 0;  // bit x: the element is an edge
+#pragma unroll
+            for (int x = 0; x < kQCols; ++x) {
+                const int u = p * 32 + x;
+                const bool in = (unsigned)(ob - omin + kDir * u) < (unsigned)orange;
+                const float bias = in ? bp[kDir * u * kQTok] : 0.f;
+                const float pr = ex2f(fmaf(__uint_as_float(sv[p][x]), rc.scale_log2e, bias));
+                float dp = __uint_as_float(dv[p][x]);
+                if constexpr (kDrop) dp *= dropout_weight(drop, rc.pair, rc.dst, src0 + (uint32_t)u);  // dP = W d_out.v; dS keeps the undropped P
+                dsv[x] = in ? pr * (dp - rc.delta) : 0.f;
+                inm |= in ? 1u << x : 0u;
+            }
+            // by-offset stores: the 8 offsets of this piece lie in at most two 16-byte chunks of the row
+            const int of = ob + kDir * (p * 32);          // offset of the thread's first column of the piece
+            const int a = of & 7, c1 = of >> 3, c2 = c1 + kDir;
+            unsigned char* b1 = rc.sk_row + ((c1 >> 3) * (kQTok * 128)) + (((c1 & 7) ^ r7) << 4) + a * 2;
+            unsigned char* b2 = rc.sk_row + ((c2 >> 3) * (kQTok * 128)) + (((c2 & 7) ^ r7) << 4) + (a - kDir * 8) * 2;
+            uint32_t pk[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) pk[x] = pack_bf16(dsv[2 * x], dsv[2 * x + 1]);
+#pragma unroll
+            for (int x = 0; x < kQCols; ++x) {
+                const bool first_chunk = kDir > 0 ? (x < 8 - a) : (x <= a);
+                if (inm & (1u << x))
+                    *reinterpret_cast<uint16_t*>((first_chunk ? b1 : b2) + kDir * x * 2) = (uint16_t)((x & 1) ? pk[x >> 1] >> 16 : pk[x >> 1] & 0xffffu);
+            }
+            const int ci = ch0 + p * 4 + rc.part;  // 16-byte chunk (8 keys) of the dS row
+            if (ci < n_ch)
+                *reinterpret_cast<uint4*>(rc.ds_s + (ci >> 3) * (kQTok * 128) + tile_off(rc.row, ci & 7)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
     }
 }
 
@@ -106,6 +165,7 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
     const int chunks = n_left + n_right;
     int2* crange = reinterpret_cast<int2*>(bnd + chunks * kQTok);
     Item* items = reinterpret_cast<Item*>(crange + chunks + (chunks & 1));  // 16-byte aligned
+    short2* wrange = reinterpret_cast<short2*>(items + kQMaxItems);           // [chunks][4]: union of the ranges of 32 rows
 
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int t0 = blockIdx.x * kQTok, h = blockIdx.y, b = blockIdx.z;
@@ -119,7 +179,7 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
     // bounded wait; once any wait has given up every later one returns at once, so the kernel winds down
     auto wait = [&](int i, uint32_t parity) {
         if (*abort_s) return;
-        if (!tc5::mbar_wait(bar(i), parity)) *abort_s = 1;
+        if (!tc5::mbar_wait_fast(bar(i), parity)) *abort_s = 1;
     };
 
     // ---- prologue: Q, d_out and out tiles, row terms, row ranges, barriers, tensor memory ----
@@ -216,6 +276,11 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
         }
         *n_items_s = n;
     }
+    for (int e = w; e < chunks * 4; e += kQThreads / 32) {  // per chunk and group of 32 rows: the union of the rows' ranges
+        const int2 a = rows_union(bnd_abs + (e >> 2) * kQTok, (e & 3) * 32, 32, lane);
+        const int base = crange[e >> 2].x;
+        if (lane == 0) wrange[e] = a.x <= a.y ? make_short2((short)(a.x - base), (short)(a.y - base)) : make_short2(1, 0);
+    }
     __syncthreads();  // also: the out tile in the dS buffer and the absolute ranges in the skew buffer are consumed
     const int J = *n_items_s;
     const int rel_cols = (t.k + 2 + 15) & ~15;  // relation rows a chunk can use, in whole 16-row boxes
@@ -256,75 +321,83 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
             }
         }
     } else if (w == kQRowThreads / 32 + 1) {
-        // =============== MMA warp: one thread issues every tensor-core instruction ===============
+        // =============== first MMA warp: one thread issues QR (first item of a chunk), S and dP of every item ===============
         if (lane == 0) {
-            int ci_a = -1, ci_b = -1;
-            auto issue_a = [&](int j) {  // QR (first item of a chunk), S and dP of item j
+            const uint32_t q_lo = tc5::desc_lo_k_major(q_u), g_lo = tc5::desc_lo_k_major(g_u), v_lo = tc5::desc_lo_k_major(v_u);
+            const uint32_t id_qr = tc5::instr_desc(kQTok, rel_cols, 0, 0);
+            int ci_a = -1;
+            for (int j = 0; j < J && !*abort_s; ++j) {
                 const Item it = items[j];
                 const int kb = j % kQKBufs, ku = j / kQKBufs;
                 if (it.flags & 1) { ++ci_a; wait(kBarRFull + (ci_a & 1), (ci_a >> 1) & 1); }
                 wait(kBarKFull + kb, ku & 1);
                 wait(kBarVFull, j & 1);
                 if (j > 0) wait(kBarSFree, (j - 1) & 1);   // every row thread holds its part of the item before
-                if (*abort_s) return;
+                if (*abort_s) break;
                 tc5::fence_after_sync();
-                const uint32_t kk_u = k_u + kb * (kQItemCols * 128);
+                const uint32_t k_lo = tc5::desc_lo_k_major(k_u + kb * (kQItemCols * 128));
                 if (it.flags & 1) {
-                    const uint32_t rr_u = r_u + (ci_a & 1) * (kQRelRows * 128);
-                    const uint32_t id_qr = tc5::instr_desc(kQTok, rel_cols, 0, 0);
+                    const uint32_t r_lo = tc5::desc_lo_k_major(r_u + (ci_a & 1) * (kQRelRows * 128));
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        tc5::mma(tbase + kQColQR, tc5::desc_k_major(q_u + ks * 32), tc5::desc_k_major(rr_u + ks * 32), id_qr, ks > 0);
+                    for (int ks = 0; ks < 4; ++ks) tc5::mma_lo(tbase + kQColQR, q_lo + ks * 2, r_lo + ks * 2, id_qr, ks > 0);
                 }
                 const uint32_t id_s = tc5::instr_desc(kQTok, it.ncols, 0, 0);
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    tc5::mma(tbase + kQColS, tc5::desc_k_major(q_u + ks * 32), tc5::desc_k_major(kk_u + ks * 32), id_s, ks > 0);
+                for (int ks = 0; ks < 4; ++ks) tc5::mma_lo(tbase + kQColS, q_lo + ks * 2, k_lo + ks * 2, id_s, ks > 0);
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks)
-                    tc5::mma(tbase + kQColDP, tc5::desc_k_major(g_u + ks * 32), tc5::desc_k_major(v_u + ks * 32), id_s, ks > 0);
+                for (int ks = 0; ks < 4; ++ks) tc5::mma_lo(tbase + kQColDP, g_lo + ks * 2, v_lo + ks * 2, id_s, ks > 0);
                 tc5::commit(bar(kBarSFull));
                 tc5::commit(bar(kBarVFree));
-            };
-            auto issue_b = [&](int j) {  // dQ += dS K_item (+ skew(dS) R_chunk with the chunk's last item)
+            }
+        }
+    } else if (w == kQRowThreads / 32 + 2) {
+        // =============== second MMA warp: one thread issues dQ += dS K_item (+ skew(dS) R_chunk with the chunk's last item) ===============
+        if (lane == 0) {
+            const uint32_t ds_lo = tc5::desc_lo_k_major(ds_u), sk_lo = tc5::desc_lo_k_major(sk_u);
+            const uint32_t id_o = tc5::instr_desc(kQTok, 64, 0, 1);
+            int ci_b = -1;
+            for (int j = 0; j < J && !*abort_s; ++j) {
                 const Item it = items[j];
                 const int kb = j % kQKBufs;
                 if (it.flags & 1) ++ci_b;
                 wait(kBarDsFull, j & 1);
-                if (*abort_s) return;
+                if (*abort_s) break;
                 tc5::fence_after_sync();
-                const uint32_t kk_u = k_u + kb * (kQItemCols * 128);
-                const uint32_t id_o = tc5::instr_desc(kQTok, 64, 0, 1);
-                for (int kk = 0; kk < (it.ncols >> 4); ++kk)
-                    tc5::mma(tbase + kQColDQ, tc5::desc_k_major(ds_u + (kk >> 2) * (kQTok * 128) + (kk & 3) * 32),
-                             tc5::desc_mn_major(kk_u + kk * 2048), id_o, (j > 0 || kk > 0) ? 1u : 0u);
+                const uint32_t k_lo = tc5::desc_lo_mn_major(k_u + kb * (kQItemCols * 128));
+                const int nk = it.ncols >> 4;
+#pragma unroll
+                for (int kk = 0; kk < kQItemCols / 16; ++kk)   // a k-step of 16 keys: 32 bytes along a dS row, 16 rows of K
+                    if (kk < nk)
+                        tc5::mma_lo(tbase + kQColDQ, ds_lo + (kk >> 2) * (kQTok * 128 / 16) + (kk & 3) * 2, k_lo + kk * (2048 / 16), id_o,
+                                    (j > 0 || kk > 0) ? 1u : 0u);
                 if (it.flags & 2) {
-                    const uint32_t rr_u = r_u + (ci_b & 1) * (kQRelRows * 128);
-                    for (int kk = 0; kk < (rel_cols >> 4); ++kk)
-                        tc5::mma(tbase + kQColDQ, tc5::desc_k_major(sk_u + (kk >> 2) * (kQTok * 128) + (kk & 3) * 32),
-                                 tc5::desc_mn_major(rr_u + kk * 2048), id_o, 1u);
+                    const uint32_t r_lo = tc5::desc_lo_mn_major(r_u + (ci_b & 1) * (kQRelRows * 128));
+                    const int nr = rel_cols >> 4;
+#pragma unroll
+                    for (int kk = 0; kk < kQRelRows / 16; ++kk)
+                        if (kk < nr)
+                            tc5::mma_lo(tbase + kQColDQ, sk_lo + (kk >> 2) * (kQTok * 128 / 16) + (kk & 3) * 2, r_lo + kk * (2048 / 16), id_o, 1u);
                     tc5::commit(bar(kBarRFree + (ci_b & 1)));
                 }
                 tc5::commit(bar(kBarKFree + kb));
                 tc5::commit(bar(kBarDsFree));
-            };
-            if (J > 0) issue_a(0);
-            for (int j = 0; j < J; ++j) {
-                if (j + 1 < J) issue_a(j + 1);
-                issue_b(j);
             }
         }
     } else {
         // =============== row threads: four per token row ===============
         const int quad = w & 3, part = w >> 2, row = quad * 32 + lane;
         const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
-        constexpr int kCols = 32 / kQTpr;  // columns of one 32-column piece a thread takes
         const float scale_log2e = scale * kLog2e;
-        const float lse_r = lse_s[row], del_r = delta_s[row];
+        RowCtx rc;
+        rc.row = row; rc.part = part;
+        rc.lse = lse_s[row]; rc.delta = delta_s[row]; rc.scale_log2e = scale_log2e;
+        rc.bias_row = bias_s + row;
+        rc.sk_row = sk_s + row * 128;
+        rc.ds_s = ds_s;
+        rc.pair = (uint32_t)(b * H + h); rc.dst = (uint32_t)(t0 + row);
         for (int j = 0; j < J; ++j) {
             const Item it = items[j];
-            int level, side, base;
-            chunk_of(it, level, side, base);
+            const int side = it.c >= n_left;
             const bool first = it.flags & 1;
             wait(kBarSFull, j & 1);   // QR (first item), S and dP of this item are in tensor memory
             tc5::fence_after_sync();
@@ -334,25 +407,20 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
             if (have_qr) tc5::tmem_ld16(tbase + lane_base + kQColQR + part * 16, qr);
             if (have_qr2) tc5::tmem_ld16(tbase + lane_base + kQColQR + 64, qr2);
 
-            // this row's columns inside the item, and the warp's union of them
+            // the columns of the item this warp's rows reach (chunk coordinates), from the table of the prologue
             const short2 my = bnd[it.c * kQTok + row];
-            const int lo_i = max((int)my.x, it.col0) - it.col0, hi_i = min((int)my.y, it.col0 + it.ncols - 1) - it.col0;
-            const bool any_i = my.x <= my.y && lo_i <= hi_i;
-            int wlo = any_i ? lo_i : 0x7fff, whi = any_i ? hi_i : -1;
-#pragma unroll
-            for (int sh = 16; sh > 0; sh >>= 1) {
-                wlo = min(wlo, __shfl_xor_sync(0xffffffffu, wlo, sh));
-                whi = max(whi, __shfl_xor_sync(0xffffffffu, whi, sh));
-            }
-            const bool w_any = wlo <= whi;
-            const int c0 = w_any ? (wlo & ~7) : 0;
-            const int npieces = w_any ? min(kQPieces, ((whi - c0) >> 5) + 1) : 0;
-            uint32_t sv[kQPieces][kCols], dv[kQPieces][kCols];
+            const short2 wu = wrange[it.c * 4 + quad];
+            const int col_end = it.col0 + it.ncols;
+            const int wlo = max((int)wu.x, it.col0), whi = min((int)wu.y, col_end - 1);
+            const bool w_any = wu.x <= wu.y && wlo <= whi;
+            const int c0 = w_any ? ((wlo - it.col0) & ~7) : 0;   // item coordinates
+            const int npieces = w_any ? min(kQPieces, ((whi - it.col0 - c0) >> 5) + 1) : 0;
+            uint32_t sv[kQPieces][kQCols], dv[kQPieces][kQCols];
 #pragma unroll
             for (int p = 0; p < kQPieces; ++p)
                 if (p < npieces) {
-                    tc5::tmem_ld8(tbase + lane_base + kQColS + c0 + p * 32 + part * kCols, sv[p]);
-                    tc5::tmem_ld8(tbase + lane_base + kQColDP + c0 + p * 32 + part * kCols, dv[p]);
+                    tc5::tmem_ld8(tbase + lane_base + kQColS + c0 + p * 32 + part * kQCols, sv[p]);
+                    tc5::tmem_ld8(tbase + lane_base + kQColDP + c0 + p * 32 + part * kQCols, dv[p]);
                 }
             tc5::tmem_ld_wait();
             tc5::fence_before_sync();
@@ -360,14 +428,15 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
 
             if (first) {
                 quad_bar(quad);  // every thread of the row group is done with the previous chunk's bias values
+                // table entry = scale * log2(e) * q.r - lse * log2(e): the exponent of an edge is one fused multiply-add away
                 if (have_qr) {
 #pragma unroll
                     for (int x = 0; x < 16; ++x)
-                        if (part * 16 + x < kQBiasRows) bias_s[(part * 16 + x) * kQTok + row] = __uint_as_float(qr[x]) * scale_log2e;
+                        if (part * 16 + x < kQBiasRows) bias_s[(part * 16 + x) * kQTok + row] = fmaf(__uint_as_float(qr[x]), scale_log2e, -rc.lse);
                 }
                 if (have_qr2) {
 #pragma unroll
-                    for (int x = 0; x < kQBiasRows - 64; ++x) bias_s[(64 + x) * kQTok + row] = __uint_as_float(qr2[x]) * scale_log2e;
+                    for (int x = 0; x < kQBiasRows - 64; ++x) bias_s[(64 + x) * kQTok + row] = fmaf(__uint_as_float(qr2[x]), scale_log2e, -rc.lse);
                 }
             }
             if (j > 0) wait(kBarDsFree, (j - 1) & 1);  // the products that read the dS tiles of the item before are done
@@ -378,41 +447,20 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
                 quad_bar(quad);  // bias values and zeros of the row are in place
             }
 
-            // the row's range in chunk coordinates: cnt nodes starting at column my.x; offset of chunk column e:
-            // right side e - my.x, left side my.y - e
+            // The row attends chunk columns my.x .. my.y (cnt of them); chunk column e has offset e - my.x on the right
+            // side and my.y - e on the left side.  This thread's first column is e0; its columns inside both the row's
+            // range and the item are those whose offset lies in [omin, omin + orange).
             const int cnt = my.x <= my.y ? my.y - my.x + 1 : 0;
-            const int e0 = it.col0 + c0 + part * kCols;          // chunk column of this thread's first column of piece 0
-            const int ch0 = c0 >> 3, n_ch = it.ncols >> 3;
-#pragma unroll
-            for (int p = 0; p < kQPieces; ++p) {
-                if (p < npieces) {
-                    uint32_t pk[4];
-                    float dsv[kCols];
-#pragma unroll
-                    for (int x = 0; x < kCols; ++x) {  // branch-free: a column outside the row's range computes on clamped indices and stores zeros
-                        const int e = e0 + p * 32 + x;
-                        const int off_raw = side ? e - my.x : my.y - e;
-                        const bool in = (unsigned)off_raw < (unsigned)cnt && e < it.col0 + it.ncols;
-                        const int off = in ? off_raw : 0;
-                        const float pr = ex2f(fmaf(__uint_as_float(sv[p][x]), scale_log2e, bias_s[off * kQTok + row]) - lse_r);
-                        float dp = __uint_as_float(dv[p][x]);
-                        if constexpr (kDrop)   // dP = W d_out.v; dS keeps the undropped P
-                            dp *= dropout_weight(drop, (uint32_t)(b * H + h), (uint32_t)(t0 + row),
-                                                 (uint32_t)(node_id(t.n, level, 0) + base + e));
-                        const float d = in ? pr * (dp - del_r) : 0.f;
-                        // column kQRelRows - 1 of the by-offset tile is no relation offset: the zeros of missing columns land there
-                        const int so = in ? off : kQRelRows - 1;
-                        *reinterpret_cast<__nv_bfloat16*>(sk_s + (so >> 6) * (kQTok * 128) + tile_off(row, (so & 63) >> 3) + (so & 7) * 2) =
-                            __float2bfloat16_rn(d);
-                        dsv[x] = d;
-                    }
-#pragma unroll
-                    for (int x = 0; x < 4; ++x) pk[x] = pack_bf16(dsv[2 * x], dsv[2 * x + 1]);
-                    const int ci = ch0 + p * 4 + part;  // 16-byte chunk (8 keys) of the dS row
-                    if (ci < n_ch)
-                        *reinterpret_cast<uint4*>(ds_s + (ci >> 3) * (kQTok * 128) + tile_off(row, ci & 7)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                }
-            }
+            const int e0 = it.col0 + c0 + part * kQCols;
+            const int n_ch = it.ncols >> 3, ch0 = c0 >> 3;
+            int ob, omin, omax1;
+            if (side) { ob = e0 - my.x; omin = 0; omax1 = min(cnt, col_end - my.x); }
+            else { ob = my.y - e0; omin = max(0, my.y - (col_end - 1)); omax1 = cnt; }
+            const int orange = max(omax1 - omin, 0);
+            uint32_t src0 = 0;
+            if constexpr (kDrop) src0 = (uint32_t)(node_id(t.n, side ? it.c - n_left : it.c, 0) + crange[it.c].x + e0);
+            if (side) q_rows_item<1, kDrop>(rc, sv, dv, npieces, ob, omin, orange, ch0, n_ch, drop, src0);
+            else q_rows_item<-1, kDrop>(rc, sv, dv, npieces, ob, omin, orange, ch0, n_ch, drop, src0);
             for (int ci = part; ci < n_ch; ci += kQTpr)  // the rest of the row is zero
                 if (ci < ch0 || ci >= ch0 + npieces * 4)
                     *reinterpret_cast<uint4*>(ds_s + (ci >> 3) * (kQTok * 128) + tile_off(row, ci & 7)) = make_uint4(0, 0, 0, 0);

@@ -43,6 +43,17 @@ __device__ __forceinline__ void mma(uint32_t d_tmem, uint64_t adesc, uint64_t bd
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}\n"
                  :: "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
 }
+// The same with the operand descriptors as (low, high) words.  The high word of every descriptor used here is
+// desc_hi() (8-row groups 1024 bytes apart, version 1, 128-byte swizzle); the low word is the start address in
+// 16-byte units plus the leading-dimension offset, so stepping through a tile is a 32-bit add on the low word.
+__device__ __forceinline__ uint32_t desc_hi() { return (1024u >> 4) | (1u << 14) | (2u << 29); }
+__device__ __forceinline__ uint32_t desc_lo_k_major(uint32_t saddr) { return ((saddr >> 4) & 0x3fff) | ((16u >> 4) << 16); }
+__device__ __forceinline__ uint32_t desc_lo_mn_major(uint32_t saddr) { return ((saddr >> 4) & 0x3fff) | ((1024u >> 4) << 16); }
+__device__ __forceinline__ void mma_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tmov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}\n"
+                 :: "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(acc), "r"(desc_hi()) : "memory");
+}
 // The mbarrier gets one arrival once every MMA this thread issued so far has completed.
 __device__ __forceinline__ void commit(uint32_t mbar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(mbar) : "memory");
@@ -63,6 +74,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t mbar, uint32_t parity, long l
                      : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
         if (ok) return true;
         if (clock64() - start > limit) return false;
+    }
+}
+// The same for the threads on the critical path of a pipeline: the clock is read every 32nd probe only.
+__device__ __forceinline__ bool mbar_wait_fast(uint32_t mbar, uint32_t parity, long long limit = kWaitCycles) {
+    long long start = 0;
+    for (uint32_t it = 0;; ++it) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                     : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((it & 31) == 31) {
+            const long long now = clock64();
+            if (start == 0) start = now;
+            else if (now - start > limit) return false;
+        }
     }
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
