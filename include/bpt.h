@@ -305,6 +305,19 @@ bpt_status bpt_trace_end(int32_t* n_marks, float* ms, const char** names, int32_
  */
 bpt_status bpt_selftest_wait_timeout(void* workspace, int64_t limit_cycles, int32_t arrive, void* cuda_stream);
 
+/*
+ * Index checks (no counterpart in the paper).  The package builds the library twice: libbpt.so, and
+ * libbpt_check.so compiled with -DBPT_BOUNDS_CHECK, in which every index a gather or an index-array
+ * write uses (an offset into col / rel / t_dst / t_eid against E, a gathered or staged node row against
+ * n_nodes, a relation row against n_rel, an edge id against E) is tested before the access.  A
+ * violation is counted, the first one recorded, and the access skipped; nothing traps.
+ * bpt_debug_bounds waits for `cuda_stream`, copies the record to `record` (host, four words:
+ * number of violations, site code of the first one, its index, its limit) and clears it.
+ * In libbpt.so the checks are compiled out and the call returns BPT_ERR_UNSUPPORTED.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+bpt_status bpt_debug_bounds(uint32_t* record, void* cuda_stream);
+
 /* Static description of a status code (host). */
 const char* bpt_status_str(bpt_status s);
 

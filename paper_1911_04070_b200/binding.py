@@ -13,6 +13,7 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libbpt.so")
+CHECK_LIB_PATH = os.path.join(_HERE, "libbpt_check.so")   # the build with index checks; set LIB_PATH to it before the first call
 
 BPT_BIDIR, BPT_LEFT_ONLY, BPT_MODE_PAD, BPT_MODE_ALG1 = 0, 1, 0, 2
 BPT_F32, BPT_BF16 = 0, 1
@@ -22,7 +23,7 @@ EXPORTS = ("bpt_graph_dims_query", "bpt_build_graph", "bpt_attn_workspace_bytes"
            "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end",
            "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch", "bpt_attn_fwd_varlen", "bpt_attn_bwd_varlen",
            "bpt_attn_fwd_ex", "bpt_attn_bwd_ex", "bpt_attn_fwd_rows", "bpt_attn_bwd_min_workspace_bytes", "bpt_check",
-           "bpt_selftest_wait_timeout")
+           "bpt_selftest_wait_timeout", "bpt_debug_bounds")
 
 
 class BptError(RuntimeError):
@@ -76,6 +77,8 @@ def load_library() -> ctypes.CDLL:
         lib.bpt_check.argtypes = [vp, vp]
         lib.bpt_selftest_wait_timeout.restype = ctypes.c_int
         lib.bpt_selftest_wait_timeout.argtypes = [vp, ctypes.c_int64, i32, vp]
+        lib.bpt_debug_bounds.restype = ctypes.c_int
+        lib.bpt_debug_bounds.argtypes = [ctypes.POINTER(ctypes.c_uint32), vp]
         lib.bpt_attn_fwd.restype = ctypes.c_int
         lib.bpt_attn_fwd.argtypes = [ctypes.POINTER(GraphStruct), i32, i32, i32, ctypes.c_int, vp, vp, vp, vp, f32,
                                      vp, vp, vp, sz, vp]
@@ -197,11 +200,19 @@ def bpt_check(workspace) -> int:
         return int(load_library().bpt_check(_ptr(workspace), _stream()))
 
 
+def bpt_debug_bounds():
+    """The index-check record of the checking build as (violations, site, index, limit); raises BptError
+    with status 2 on the normal build, which carries no checks."""
+    rec = (ctypes.c_uint32 * 4)()
+    _check(load_library().bpt_debug_bounds(rec, _stream()), "bpt_debug_bounds")
+    return tuple(int(x) for x in rec)
+
+
 def bpt_selftest_wait_timeout(workspace, limit_cycles: int, arrive: bool):
     """Launches the library's wait self-test (see include/bpt.h); read the outcome with bpt_check."""
     with torch.cuda.device(workspace.device):
         _check(load_library().bpt_selftest_wait_timeout(_ptr(workspace), int(limit_cycles), int(arrive), _stream()),
-               "bpt_selftest_wait_timeout")
+               "bpt_selftest_wait_timeout", "bpt_debug_bounds")
 
 
 def _check_layout(g: Graph, q, *same):

@@ -1,5 +1,12 @@
 // C-ABI entry points: argument validation and dispatch.  See include/bpt.h.
+#include "bounds_check.cuh"
 #include "bpt_internal.cuh"
+
+#ifdef BPT_BOUNDS_CHECK
+namespace bpt {
+__device__ unsigned int g_bounds_record[4];
+}
+#endif
 
 using namespace bpt;
 
@@ -212,6 +219,19 @@ extern "C" bpt_status bpt_trace_end(int32_t* n_marks, float* ms, const char** na
     *n_marks = n < 0 ? 0 : n;
     g_trace.n = g_trace.cap = 0;
     return st;
+}
+
+extern "C" bpt_status bpt_debug_bounds(uint32_t* record, void* cuda_stream) {
+#ifdef BPT_BOUNDS_CHECK
+    if (!record) return BPT_ERR_INVALID_ARG;
+    if (cudaStreamSynchronize((cudaStream_t)cuda_stream) != cudaSuccess) return BPT_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(record, g_bounds_record, sizeof(g_bounds_record)) != cudaSuccess) return BPT_ERR_CUDA;
+    const unsigned int zero[4] = {0, 0, 0, 0};
+    return cudaMemcpyToSymbol(g_bounds_record, zero, sizeof(zero)) == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
+#else
+    (void)record; (void)cuda_stream;
+    return BPT_ERR_UNSUPPORTED;   // this build carries no index checks
+#endif
 }
 
 extern "C" const char* bpt_status_str(bpt_status s) {

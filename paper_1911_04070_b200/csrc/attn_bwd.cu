@@ -9,6 +9,7 @@
 // The rows of d_rel that belong to the ancestor relations are written as exact zeros:
 // every edge into a span carries the same relation, so its embedding shifts all scores of
 // the row alike and the softmax does not depend on it.
+#include "bounds_check.cuh"
 #include "bpt_internal.cuh"
 #include "row_map.cuh"
 
@@ -53,7 +54,7 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
                const T* __restrict__ out, const float* __restrict__ lse, const T* __restrict__ d_out,
                T* __restrict__ dq, float* __restrict__ ws_p, float* __restrict__ ws_ds,
                int N, int row0, int nrows, int H, int ngroups, int64_t e_first, int64_t E, float scale,
-               const int32_t* __restrict__ lengths, DropoutParams drop) {
+               const int32_t* __restrict__ lengths, DropoutParams drop, int n_rel) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
@@ -95,7 +96,7 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
     for (int e0 = a + w * U; e0 < z; e0 += nw * U) {
         const int cnt = min(U, z - e0);
         int my_c = 0, my_r = 0;
-        if (lane < cnt) { my_c = col[e0 + lane]; my_r = rel[e0 + lane]; }
+        if (lane < cnt && BPT_IDX_OK(e0 + lane, E, BPT_SITE_CSR_OFFSET)) { my_c = col[e0 + lane]; my_r = rel[e0 + lane]; }
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             const int c = __shfl_sync(0xffffffffu, my_c, j), rr = __shfl_sync(0xffffffffu, my_r, j);
@@ -105,7 +106,7 @@ bwd_dst_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ 
                     ws_p[o] = 0.f;
                     ws_ds[o] = 0.f;
                 }
-            } else if (j < cnt) {  // uniform over the warp
+            } else if (j < cnt && BPT_IDX_OK(c, N, BPT_SITE_NODE) && BPT_IDX_OK(rr, n_rel, BPT_SITE_RELATION)) {  // uniform over the warp
                 float kk[EPL], rv[EPL], vv[EPL];
                 M::load(k + boff + (size_t)c * rs, sub, kk);
                 M::load(r + (size_t)rr * D, sub, rv);
@@ -185,11 +186,11 @@ bwd_src_kernel(const int32_t* __restrict__ t_ptr, const int32_t* __restrict__ t_
     for (int e0 = a + w * U; e0 < z; e0 += nw * U) {
         const int cnt = min(U, z - e0);
         int my_u = 0, my_e = 0;
-        if (lane < cnt) { my_u = t_dst[e0 + lane]; my_e = t_eid[e0 + lane]; }
+        if (lane < cnt && BPT_IDX_OK(e0 + lane, E, BPT_SITE_CSR_OFFSET)) { my_u = t_dst[e0 + lane]; my_e = t_eid[e0 + lane]; }
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             const int u = __shfl_sync(0xffffffffu, my_u, j), e = __shfl_sync(0xffffffffu, my_e, j);
-            if (j < cnt) {
+            if (j < cnt && BPT_IDX_OK(u, N, BPT_SITE_NODE) && BPT_IDX_OK(e, E, BPT_SITE_EDGE_ID)) {
                 float qv[EPL], gv[EPL];
                 M::load(q + boff + (size_t)u * rs, sub, qv);
                 M::load(d_out + boff + (size_t)u * rs, sub, gv);
@@ -379,7 +380,7 @@ static bpt_status launch_bwd_rows(const AttnProblem& p) {
     const size_t smem_a = nw > 1 ? (size_t)nw * 32 * M::EPL * sizeof(float) : 0;
     bwd_dst_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem_a, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, 0, N, p.H, ngroups, 0, E, p.scale, p.lengths, p.drop);
+        (const T*)p.out, p.lse, (const T*)p.d_out, (T*)p.dq, ws.p, ws.ds, N, 0, N, p.H, ngroups, 0, E, p.scale, p.lengths, p.drop, g.dims.n_rel);
     trace_mark(p.stream, "bwd_dst");
 
     const size_t smem_b = nw > 1 ? (size_t)nw * 32 * (2 * M::EPL) * sizeof(float) : 0;

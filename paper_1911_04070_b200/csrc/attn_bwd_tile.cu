@@ -18,6 +18,7 @@
 // Nothing is accumulated across CTAs here: bwd_gather_kernel sums, for every source node, the
 // partial rows of the tiles whose range covers it, in tile order (no atomics, fixed order), and
 // drel_sum kernels do the same for the relation table.
+#include "bounds_check.cuh"
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
 #include "row_map.cuh"
@@ -228,13 +229,15 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
             const int row = idx >> 3, ch = idx & 7;
             const int node = min(gm.base + s0 + row, gm.n_l - 1);  // rows past the range repeat a real row: finite values
             const size_t src = boff + (size_t)(gm.id_base + node) * rs + ch * 8;
+            if (!BPT_IDX_OK(gm.id_base + node, N, BPT_SITE_NODE)) continue;
             cp_async16(k_u + tile_off(row, ch), k + src);
             cp_async16(v_u + tile_off(row, ch), v + src);
         }
         if (s0 == 0) {
             for (int idx = tid; idx < cfg.rel_rows * 8; idx += kBwdThreads) {
                 const int row = idx >> 3, ch = idx & 7;
-                if (row < gm.n_rel_c) cp_async16(r_u + tile_off(row, ch), r + (size_t)(gm.rel_base + row) * 64 + ch * 8);
+                if (row < gm.n_rel_c && BPT_IDX_OK(gm.rel_base + row, 1 + 2 * t.L * (t.k + 1) + t.L, BPT_SITE_RELATION))
+                    cp_async16(r_u + tile_off(row, ch), r + (size_t)(gm.rel_base + row) * 64 + ch * 8);
                 else *reinterpret_cast<uint4*>(r_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
             }
         }

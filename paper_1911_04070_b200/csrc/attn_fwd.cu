@@ -4,6 +4,7 @@
 // registers, and the per-warp states are merged in a fixed order through shared memory.
 #include <cstdlib>
 
+#include "bounds_check.cuh"
 #include "bpt_internal.cuh"
 #include "row_map.cuh"
 #include "tile_geom.cuh"
@@ -19,7 +20,7 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
                 const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v, const T* __restrict__ r,
                 T* __restrict__ out, float* __restrict__ lse, int N, int row0, int nrows, int H, int ngroups,
                 float scale_log2e, const int32_t* __restrict__ lengths, DropoutParams drop,
-                const int32_t* __restrict__ row_list) {
+                const int32_t* __restrict__ row_list, int64_t E, int n_rel) {
     using M = RowMap<T, D>;
     constexpr int EPL = M::EPL;
     extern __shared__ float smem[];
@@ -54,13 +55,14 @@ fwd_rows_kernel(const int32_t* __restrict__ row_ptr, const int32_t* __restrict__
     for (int e0 = a + w * U; e0 < z; e0 += nw * U) {
         const int cnt = min(U, z - e0);
         int my_c = 0, my_r = 0;
-        if (lane < cnt) { my_c = col[e0 + lane]; my_r = rel[e0 + lane]; }
+        if (lane < cnt && BPT_IDX_OK(e0 + lane, E, BPT_SITE_CSR_OFFSET)) { my_c = col[e0 + lane]; my_r = rel[e0 + lane]; }
         float s[U], vv[U][EPL], wgt[U];
 #pragma unroll
         for (int j = 0; j < U; ++j) {
             const int c = __shfl_sync(0xffffffffu, my_c, j), rr = __shfl_sync(0xffffffffu, my_r, j);
             wgt[j] = (drop.thr && j < cnt) ? dropout_weight(drop, (uint32_t)(b * H + hc), (uint32_t)u, (uint32_t)c) : 1.f;
-            if (j < cnt && (len >= n_tok || node_first_token(n_tok, c) < len)) {
+            if (j < cnt && BPT_IDX_OK(c, N, BPT_SITE_NODE) && BPT_IDX_OK(rr, n_rel, BPT_SITE_RELATION) &&
+                (len >= n_tok || node_first_token(n_tok, c) < len)) {
                 float kk[EPL], rv[EPL];
                 M::load(k + boff + (size_t)c * rs, sub, kk);
                 M::load(r + (size_t)rr * D, sub, rv);
@@ -148,7 +150,7 @@ static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows, const i
     const size_t smem = nw > 1 ? (size_t)nw * 32 * (2 + M::EPL) * sizeof(float) : 0;
     fwd_rows_kernel<T, D, U><<<(unsigned)blocks, nw * 32, smem, p.stream>>>(
         g.row_ptr, g.col, g.rel, (const T*)p.q, (const T*)p.k, (const T*)p.v, (const T*)p.rel_emb,
-        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e, p.lengths, p.drop, row_list);
+        (T*)p.out, p.lse, N, row0, nrows, p.H, ngroups, p.scale * kLog2e, p.lengths, p.drop, row_list, g.dims.n_edges, g.dims.n_rel);
     trace_mark(p.stream, "fwd_rows");
     return cudaGetLastError() == cudaSuccess ? BPT_OK : BPT_ERR_CUDA;
 }

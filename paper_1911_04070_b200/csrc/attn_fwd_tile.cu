@@ -10,6 +10,7 @@
 // q_i . r[rel(i, m)] depends on the offset of node m inside token i's range: the warp
 // computes Q R_chunk^T once per chunk (a dense 16 x (k+1) product), parks it in shared
 // memory and every score picks its entry by offset.
+#include "bounds_check.cuh"
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
 #include "tile_geom.cuh"
@@ -171,12 +172,13 @@ fwd_tile_kernel(TreeParams t, FwdTileCfg cfg, int n_left, int n_right,
             const int row = idx >> 3, ch = idx & 7;
             const int node = min(base + row, n_l - 1);
             const size_t src = boff + (size_t)(id_base + node) * rs + ch * 8;
+            if (!BPT_IDX_OK(id_base + node, 2 * t.n - 1, BPT_SITE_NODE)) continue;
             cp_async16(k_u + tile_off(row, ch), k + src);
             cp_async16(v_u + tile_off(row, ch), v + src);
         }
         for (int idx = tid; idx < cfg.rel_rows * 8; idx += 128) {
             const int row = idx >> 3, ch = idx & 7;
-            if (row < W) cp_async16(r_u + tile_off(row, ch), r + (size_t)(rel_base + row) * 64 + ch * 8);
+            if (row < W && BPT_IDX_OK(rel_base + row, 1 + 2 * t.L * (t.k + 1) + t.L, BPT_SITE_RELATION)) cp_async16(r_u + tile_off(row, ch), r + (size_t)(rel_base + row) * 64 + ch * 8);
             else *reinterpret_cast<uint4*>(r_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
         }
         cp_async_commit();

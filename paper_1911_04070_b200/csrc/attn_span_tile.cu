@@ -10,6 +10,7 @@
 // the backward) that a small merge kernel combines over the tiles in tile order.  In the
 // backward the tile also produces, for its 64 tokens, the complete contribution of all spans
 // to dk and dv (a [64][128] fp32 block that the source-side gather adds).
+#include "bounds_check.cuh"
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
 #include "row_map.cuh"
@@ -95,7 +96,7 @@ fwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
     __syncthreads();
     for (int idx = tid; idx < kSpanRows * 8; idx += kSpanThreads) {
         const int row = idx >> 3, ch = idx & 7;
-        if (meta.node[row] >= 0) cp_async16(qs_u + tile_off(row, ch), q + boff + (size_t)meta.node[row] * rs + ch * 8);
+        if (meta.node[row] >= 0 && BPT_IDX_OK(meta.node[row], N, BPT_SITE_NODE)) cp_async16(qs_u + tile_off(row, ch), q + boff + (size_t)meta.node[row] * rs + ch * 8);
         else *reinterpret_cast<uint4*>(qs_s + tile_off(row, ch)) = make_uint4(0, 0, 0, 0);
     }
     for (int idx = tid; idx < kTileTokens * 8; idx += kSpanThreads) {
@@ -331,7 +332,7 @@ bwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
     __syncthreads();
     for (int idx = tid; idx < kSpanRows * 8; idx += kSpanThreads) {
         const int row = idx >> 3, ch = idx & 7;
-        if (meta.node[row] >= 0) {
+        if (meta.node[row] >= 0 && BPT_IDX_OK(meta.node[row], N, BPT_SITE_NODE)) {
             const size_t src = boff + (size_t)meta.node[row] * rs + ch * 8;
             cp_async16(qs_u + tile_off(row, ch), q + src);
             cp_async16(gs_u + tile_off(row, ch), d_out + src);

@@ -1,6 +1,7 @@
 // Device-side builder of the BPT attention graph (arXiv 1911.04070, Sec. 3.2.2
 // affiliated + contextual edges, Sec. 3.4 relation labels): CSR by destination and
 // the by-source lists, bit-exact and without atomics.
+#include "bounds_check.cuh"
 #include "bpt_internal.cuh"
 
 namespace bpt {
@@ -68,7 +69,7 @@ __global__ void span_row_ptr_kernel(TreeParams t, int32_t* __restrict__ row_ptr)
 // ---------------------------------------------------------------------------------
 // One warp per token row.
 __global__ void token_fill_kernel(TreeParams t, const int32_t* __restrict__ row_ptr,
-                                  int32_t* __restrict__ col, int32_t* __restrict__ rel) {
+                                  int32_t* __restrict__ col, int32_t* __restrict__ rel, int64_t E) {
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (i >= t.n) return;
@@ -79,17 +80,19 @@ __global__ void token_fill_kernel(TreeParams t, const int32_t* __restrict__ row_
     for (int l = 0; lw.valid() || (use_r && rw.valid()) || l == 0; ++l) {
         if (lw.valid()) {
             const int c = lw.hi - lw.lo + 1, base = node_id(t.n, l, lw.lo), r0 = rel_left(t, l, 0);
-            for (int j = lane; j < c; j += 32) { col[at + j] = base + j; rel[at + j] = r0 + (c - 1 - j); }
+            for (int j = lane; j < c; j += 32)
+                if (BPT_IDX_OK(at + j, E, BPT_SITE_GRAPH_WRITE)) { col[at + j] = base + j; rel[at + j] = r0 + (c - 1 - j); }
             at += c;
             lw.next();
         }
         if (l == 0) {
-            if (lane == 0) { col[at] = i; rel[at] = 0; }
+            if (lane == 0 && BPT_IDX_OK(at, E, BPT_SITE_GRAPH_WRITE)) { col[at] = i; rel[at] = 0; }
             ++at;
         }
         if (use_r && rw.valid()) {
             const int c = rw.hi - rw.lo + 1, base = node_id(t.n, l, rw.lo), r0 = rel_right(t, l, 0);
-            for (int j = lane; j < c; j += 32) { col[at + j] = base + j; rel[at + j] = r0 + j; }
+            for (int j = lane; j < c; j += 32)
+                if (BPT_IDX_OK(at + j, E, BPT_SITE_GRAPH_WRITE)) { col[at + j] = base + j; rel[at + j] = r0 + j; }
             at += c;
             rw.next();
         }
@@ -98,11 +101,12 @@ __global__ void token_fill_kernel(TreeParams t, const int32_t* __restrict__ row_
 
 // Affiliated edges: inside level l the j-th edge comes from token j.
 __global__ void span_fill_kernel(TreeParams t, const int32_t* __restrict__ row_ptr,
-                                 int32_t* __restrict__ col, int32_t* __restrict__ rel) {
+                                 int32_t* __restrict__ col, int32_t* __restrict__ rel, int64_t E) {
     const int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (x >= (int64_t)t.L * t.n) return;
     const int l = (int)(x / t.n) + 1, j = (int)(x % t.n);
     const int64_t e = (int64_t)row_ptr[t.n] + x;
+    if (!BPT_IDX_OK(e, E, BPT_SITE_GRAPH_WRITE)) return;
     col[e] = j;
     rel[e] = rel_anc(t, l);
 }
@@ -195,7 +199,7 @@ __global__ void source_degree_kernel(TreeParams t, int32_t* __restrict__ t_ptr) 
 
 // One warp per source node; destinations ascending.
 __global__ void source_fill_kernel(TreeParams t, const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ t_ptr,
-                                   int32_t* __restrict__ t_dst, int32_t* __restrict__ t_eid) {
+                                   int32_t* __restrict__ t_dst, int32_t* __restrict__ t_eid, int64_t E) {
     const int v = (int)(((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
     const int lane = threadIdx.x & 31;
     if (v >= 2 * t.n - 1) return;
@@ -206,6 +210,7 @@ __global__ void source_fill_kernel(TreeParams t, const int32_t* __restrict__ row
     for (int i = f.ra + lane; i < f.rb; i += 32) {
         int pos, cnt, first;
         token_block(t, i, 1, l, &pos, &cnt, &first);
+        if (!BPT_IDX_OK(at + i - f.ra, E, BPT_SITE_GRAPH_WRITE)) continue;
         t_dst[at + i - f.ra] = i;
         t_eid[at + i - f.ra] = row_ptr[i] + pos + (m - first);
     }
@@ -214,14 +219,17 @@ __global__ void source_fill_kernel(TreeParams t, const int32_t* __restrict__ row
         if (lane == 0) {
             int pos, cnt, first;
             token_block(t, m, 2, 0, &pos, &cnt, &first);
-            t_dst[at] = m;
-            t_eid[at] = row_ptr[m] + pos;
+            if (BPT_IDX_OK(at, E, BPT_SITE_GRAPH_WRITE)) {
+                t_dst[at] = m;
+                t_eid[at] = row_ptr[m] + pos;
+            }
         }
         ++at;
     }
     for (int i = f.la + lane; i < f.lb; i += 32) {
         int pos, cnt, first;
         token_block(t, i, 0, l, &pos, &cnt, &first);
+        if (!BPT_IDX_OK(at + i - f.la, E, BPT_SITE_GRAPH_WRITE)) continue;
         t_dst[at + i - f.la] = i;
         t_eid[at + i - f.la] = row_ptr[i] + pos + (m - first);
     }
@@ -229,6 +237,7 @@ __global__ void source_fill_kernel(TreeParams t, const int32_t* __restrict__ row
     if (l == 0) {
         for (int j = 1 + lane; j <= t.L; j += 32) {
             const int u = node_id(t.n, j, m >> j);
+            if (!BPT_IDX_OK(at + j - 1, E, BPT_SITE_GRAPH_WRITE)) continue;
             t_dst[at + j - 1] = u;
             t_eid[at + j - 1] = row_ptr[u] + (m & ((1 << j) - 1));
         }
@@ -289,15 +298,15 @@ extern "C" bpt_status bpt_build_graph(const bpt_graph_dims* dims, int32_t* row_p
     token_degree_kernel<<<(n + 255) / 256, 256, 0, st>>>(t, row_ptr);
     exclusive_scan_kernel<<<1, 1024, 0, st>>>(row_ptr, n);
     span_row_ptr_kernel<<<(n + 255) / 256, 256, 0, st>>>(t, row_ptr);
-    token_fill_kernel<<<(n * 32 + 255) / 256, 256, 0, st>>>(t, row_ptr, col, rel);
+    token_fill_kernel<<<(n * 32 + 255) / 256, 256, 0, st>>>(t, row_ptr, col, rel, dims->n_edges);
     {
         const int64_t tot = (int64_t)t.L * n;
-        span_fill_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(t, row_ptr, col, rel);
+        span_fill_kernel<<<(unsigned)((tot + 255) / 256), 256, 0, st>>>(t, row_ptr, col, rel, dims->n_edges);
     }
     if (want_t) {
         source_degree_kernel<<<(N + 127) / 128, 128, 0, st>>>(t, t_ptr);
         exclusive_scan_kernel<<<1, 1024, 0, st>>>(t_ptr, N);
-        source_fill_kernel<<<(unsigned)(((int64_t)N * 32 + 255) / 256), 256, 0, st>>>(t, row_ptr, t_ptr, t_dst, t_eid);
+        source_fill_kernel<<<(unsigned)(((int64_t)N * 32 + 255) / 256), 256, 0, st>>>(t, row_ptr, t_ptr, t_dst, t_eid, dims->n_edges);
     }
     if (cudaGetLastError() != cudaSuccess) return BPT_ERR_CUDA;
     out->row_ptr = row_ptr; out->col = col; out->rel = rel;

@@ -104,3 +104,64 @@ class BPTEncoder(nn.Module):
         if readout == "root":
             return h[:, -1]
         raise ValueError("readout must be 'tokens' or 'root'")
+
+
+class BPTDecoder:
+    """Step-by-step evaluation of a left-only BPTEncoder with cached per-layer state, for autoregressive use
+    (Sec. 4.2 trains BPT as a language model; generation feeds it one token at a time).
+
+    When token i arrives, the only nodes whose state changes in any layer are token i and its log2(n)
+    ancestors: every other token lies to its left and attends only nodes that lie wholly to its own left.
+    The decoder therefore keeps, per layer, the input states of all 2n-1 nodes and their key / value
+    rows, recomputes those log2(n) + 1 rows per layer with `bpt_attn_fwd_rows` and lengths = i + 1 (the
+    ancestors then attend exactly the tokens seen so far), and returns the last layer's state of token i.
+    A span is complete once its last token has arrived; from then on its cached state is the one a full
+    forward pass over the finished sequence computes, so the token outputs of the steps equal the token
+    rows of `BPTEncoder.forward` on the whole sequence."""
+
+    def __init__(self, enc: BPTEncoder, batch: int, dtype=torch.float32):
+        g = enc.g
+        if not (g.dims.flags & binding.BPT_LEFT_ONLY):
+            raise ValueError("step-by-step decoding needs the left-only graph")
+        self.enc, self.g, self.n, self.batch = enc, g, enc.n, batch
+        first = enc.layers[0]
+        dev = first.rel_emb.device
+        D, H, dh, N = first.h * first.dh, first.h, first.dh, g.n_nodes
+        self.L = g.dims.n_levels
+        self.h = [torch.zeros(batch, N, D, device=dev, dtype=dtype) for _ in range(len(enc.layers) + 1)]
+        heads = lambda: torch.zeros(batch, N, H, dh, device=dev, dtype=dtype)
+        self.q, self.k, self.v, self.a = ([heads() for _ in enc.layers] for _ in range(4))
+        self.lse = torch.zeros(batch, N, H, device=dev, dtype=torch.float32)
+        self.pos = 0
+
+    def rows_of_step(self, i: int):
+        """Token i and its ancestors, finest first."""
+        n = self.n
+        return [i] + [2 * n - ((2 * n) >> j) + (i >> j) for j in range(1, self.L + 1)]
+
+    @torch.no_grad()
+    def step(self, token_state):
+        """token_state: [batch, D], the input state of the next token.  Returns its output state [batch, D]."""
+        i = self.pos
+        if i >= self.n:
+            raise ValueError("the sequence is full (n = %d)" % self.n)
+        rows = self.rows_of_step(i)
+        B, R = self.batch, len(rows)
+        dev = self.h[0].device
+        idx = torch.tensor(rows, device=dev)
+        rows_t = torch.tensor([rows] * B, dtype=torch.int32, device=dev)
+        lens = torch.full((B,), i + 1, dtype=torch.int32, device=dev)
+        self.h[0][:, i] = token_state.to(self.h[0].dtype)
+        for li, layer in enumerate(self.enc.layers):
+            hr = self.h[li][:, idx]                                     # [B, R, D]; span rows of layer 0 are zero
+            split = lambda x: x.view(B, R, layer.h, layer.dh)
+            self.q[li][:, idx] = split(layer.wq(hr))
+            self.k[li][:, idx] = split(layer.wk(hr))
+            self.v[li][:, idx] = split(layer.wv(hr))
+            binding.bpt_attn_fwd_rows(self.g, self.q[li], self.k[li], self.v[li], layer.rel_emb.to(hr.dtype).contiguous(),
+                                      1.0 / math.sqrt(layer.dh), rows_t, self.a[li], self.lse, lengths=lens)
+            a = self.a[li][:, idx].reshape(B, R, -1)
+            z = layer.norm1(hr + layer.wo(a))
+            self.h[li + 1][:, idx] = layer.norm2(z + layer.ff2(torch.relu(layer.ff1(z))))
+        self.pos += 1
+        return self.h[-1][:, i]
