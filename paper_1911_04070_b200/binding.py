@@ -212,7 +212,7 @@ def bpt_selftest_wait_timeout(workspace, limit_cycles: int, arrive: bool):
     """Launches the library's wait self-test (see include/bpt.h); read the outcome with bpt_check."""
     with torch.cuda.device(workspace.device):
         _check(load_library().bpt_selftest_wait_timeout(_ptr(workspace), int(limit_cycles), int(arrive), _stream()),
-               "bpt_selftest_wait_timeout", "bpt_debug_bounds")
+               "bpt_selftest_wait_timeout")
 
 
 def _check_layout(g: Graph, q, *same):

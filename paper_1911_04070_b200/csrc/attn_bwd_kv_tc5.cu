@@ -73,39 +73,6 @@ __device__ __forceinline__ float ex2f(float x) {
     return y;
 }
 
-// Range of nodes token i attends at (side, level) with the conventions of fill_row_bounds: empty ranges
-// keep both bounds monotone in i, and the self loop joins the left range of level 0.
-__device__ __forceinline__ int2 level_range(const TreeParams& t, int i, int side, int level) {
-    if (side == 0) {
-        LeftWalk w(t, i);
-        for (int l = 0; l < level && w.valid(); ++l) w.next();
-        int2 v = w.valid() ? make_int2(w.lo, w.hi) : make_int2(0, -1);
-        if (level == 0) v = v.x > v.y ? make_int2(i, i) : make_int2(v.x, i);
-        return v;
-    }
-    RightWalk w(t, i);
-    for (int l = 0; l < level && w.valid(); ++l) w.next();
-    const int n_l = t.n >> level;
-    return w.valid() ? make_int2(w.lo, w.hi) : make_int2(n_l, n_l - 1);
-}
-
-// First i in [0, n) for which the monotone predicate holds (n if none); the whole warp calls it.
-template <typename F>
-__device__ __forceinline__ int warp_first(int n, int lane, F pred) {
-    int lo = 0, hi = n;  // the answer lies in [lo, hi]
-    while (lo < hi) {
-        const int step = (hi - lo + 31) / 32;
-        const int i = lo + lane * step;
-        const bool p = i < hi ? pred(i) : true;
-        const unsigned m = __ballot_sync(0xffffffffu, p);
-        const int f = __ffs(m) - 1;  // lanes at or beyond hi vote true, so f >= 0 unless all 32 probes are below hi and false
-        if (f < 0) { lo = lo + 31 * step + 1; continue; }
-        hi = min(hi, lo + f * step);
-        lo = f > 0 ? lo + (f - 1) * step + 1 : lo;
-    }
-    return lo;
-}
-
 // (level, first node) of key tile `x` when the tiles are numbered from the coarsest level down
 __device__ __forceinline__ void tile_of(int n, int L, int x, int* level, int* m0) {
     for (int l = L; l >= 0; --l) {
@@ -114,6 +81,30 @@ __device__ __forceinline__ void tile_of(int n, int L, int x, int* level, int* m0
         x -= tiles;
     }
     *level = 0; *m0 = 0;
+}
+
+// plan[x * 2 + side] = (first query token rounded down to a block, number of 64-token blocks) of key tile x: the
+// tokens that reach keys m0 .. m0 + 127 of the tile's level from that side form one interval, because the first
+// and the last node of a token's range grow with the token index (bisection on the table of ranges).
+__global__ void key_tile_plan_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__ ranges,
+                                     int2* __restrict__ plan, int tiles_total) {
+    const int id = blockIdx.x * blockDim.x + threadIdx.x;
+    if (id >= tiles_total * 2) return;
+    const int side = id & 1;
+    int level, m0;
+    tile_of(t.n, t.L, id >> 1, &level, &m0);
+    int2 out = make_int2(0, 0);
+    if (level < (side ? n_right : n_left)) {
+        const int2* rg = ranges + (size_t)(side ? n_left + level : level) * t.n;
+        const int m1 = m0 + kKvKeys - 1;
+        int lo = 0, hi = t.n;   // first token whose range ends at or beyond m0
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (__ldg(rg + mid).y >= m0) hi = mid; else lo = mid + 1; }
+        const int first = lo;
+        hi = t.n;               // first token whose range starts beyond m1
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (__ldg(rg + mid).x > m1) hi = mid; else lo = mid + 1; }
+        if (first < lo) { out.x = first & ~(kKvQB - 1); out.y = (lo - out.x + kKvQB - 1) / kKvQB; }
+    }
+    plan[id] = out;
 }
 
 // One item's share of a row thread: its key node m against kKvCols query columns.  Predicated, no branch per element.
@@ -161,7 +152,7 @@ __device__ __forceinline__ void kv_rows_item(const uint32_t (&sv)[kKvCols], cons
 
 template <bool kDrop>
 __global__ void __launch_bounds__(kKvThreads, 1)
-bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
+bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__ ranges, const int2* __restrict__ plan,
                   const float* __restrict__ lse, const float* __restrict__ delta_in, const float* __restrict__ aff_slab,
                   __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv, float* __restrict__ drel_part,
                   int* __restrict__ status, int H, int pair0, float scale, const int32_t* __restrict__ lengths, DropoutParams drop,
@@ -213,16 +204,9 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
         *abort_s = 0;
     }
     if (w == 0) tc5::tmem_alloc(smem_u32(tmem_slot), kKvTmemCols);
-    if (w == 1 || w == 2) {  // tokens that reach keys m0 .. m0 + 127 from the side
-        const int side = w - 1;
-        int qa = 0, nb = 0;
-        if (side_on[side]) {
-            const int m1 = m0 + kKvKeys - 1;
-            const int first = warp_first(t.n, lane, [&](int i) { return level_range(t, i, side, level).y >= m0; });
-            const int last = warp_first(t.n, lane, [&](int i) { return level_range(t, i, side, level).x > m1; });
-            if (first < last) { qa = first & ~(kKvQB - 1); nb = (last - qa + kKvQB - 1) / kKvQB; }
-        }
-        if (lane == 0) { plan_s[2 * side] = qa; plan_s[2 * side + 1] = nb; }
+    if (tid < 2) {  // the query blocks of the two sides
+        const int2 pq = __ldg(plan + (size_t)blockIdx.y * 2 + tid);
+        plan_s[2 * tid] = pq.x; plan_s[2 * tid + 1] = pq.y;
     }
     for (int idx = tid; idx < 2 * kKvKeys * 8; idx += kKvThreads)  // both by-offset tiles start from zero
         *reinterpret_cast<uint4*>(sk_s + idx * 16) = make_uint4(0, 0, 0, 0);
@@ -269,18 +253,20 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
                         tc5::tma_load_4d(g_u + rb * (kKvQB * 128) + x * 2048, &tm_g, 0, h, q0 + 16 * x, b, bar(kvQFull + rb));
                     }
                 }
-                // per query: node range at this level, lse and row term (the two loads fly while the ranges are walked)
+                // per query: node range at this level (from the table), lse and row term
                 float lv[kKvQB / 32], dl[kKvQB / 32];
+                int2 rgv[kKvQB / 32];
 #pragma unroll
                 for (int x = 0; x < kKvQB / 32; ++x) {
                     const int i = q0 + lane + 32 * x;
+                    rgv[x] = __ldg(ranges + (size_t)(side ? n_left + level : level) * t.n + i);
                     lv[x] = __ldg(lse + ((size_t)b * N_nodes + i) * H + h);
                     dl[x] = __ldg(delta_in + (size_t)pair * t.n + i);
                 }
 #pragma unroll
                 for (int x = 0; x < kKvQB / 32; ++x) {
                     const int i = q0 + lane + 32 * x;
-                    int2 rg = level_range(t, i, side, level);
+                    int2 rg = rgv[x];
                     if (len < t.n) {  // short sequence: a placeholder token attends nothing, right ranges end at the last real node
                         if (i >= len) rg = make_int2(1, 0);
                         else if (side == 1) rg.y = min(rg.y, (len - 1) >> level);
@@ -379,7 +365,6 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
                     bias[(part * kKvCols + x) * kKvBiasStride + row] = fmaf(__uint_as_float(qr[x]), scale_log2e, nl[x]);
             }
             asm volatile("bar.sync 1, %0;" ::"n"(kKvRowThreads) : "memory");  // the table of this item is complete (and the other by-offset tile is cleared)
-            if (j > 0) wait(kvDsFree, (j - 1) & 1);   // the products that read P^T, dS^T of the item before are done
 
             // does any of the warp's 32 keys meet any of this thread group's 16 queries?
             bool hit = false;
@@ -393,6 +378,7 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right,
                 if (side) kv_rows_item<1, kDrop>(sv, dv, mq, bias_col, skw, m, part, scale_log2e, drop, (uint32_t)pair, dst0, src, pp, dd);
                 else kv_rows_item<0, kDrop>(sv, dv, mq, bias_col, skw, m, part, scale_log2e, drop, (uint32_t)pair, dst0, src, pp, dd);
             }
+            if (j > 0) wait(kvDsFree, (j - 1) & 1);   // the products that read P^T, dS^T of the item before are done (hidden behind the weights above)
 #pragma unroll
             for (int c = 0; c < kKvCols / 8; ++c) {
                 *reinterpret_cast<uint4*>(p_s + tile_off(row, part * (kKvCols / 8) + c)) = make_uint4(pp[4 * c], pp[4 * c + 1], pp[4 * c + 2], pp[4 * c + 3]);
@@ -539,7 +525,8 @@ size_t bwd_kv_tc5_drel_floats(const TreeParams& t, int n_pairs) {
 }
 
 // dk, dv of all nodes of pairs [pair0, pair0 + n_pairs) and d_rel (added to with pair0 > 0).
-bpt_status launch_bwd_kv_tc5(const AttnProblem& p, int pair0, int n_pairs, const float* delta, const float* aff_slab, float* drel_part) {
+bpt_status launch_bwd_kv_tc5(const AttnProblem& p, int pair0, int n_pairs, const float* delta, const int2* ranges, int2* plan,
+                             const float* aff_slab, float* drel_part) {
     const TreeParams& t = p.tree;
     int n_left, n_right;
     context_levels(t, &n_left, &n_right);
@@ -552,8 +539,12 @@ bpt_status launch_bwd_kv_tc5(const AttnProblem& p, int pair0, int n_pairs, const
         !tc5::rel_rows_map(&tm_r, p.rel_emb, p.g->dims.n_rel))
         return BPT_ERR_CUDA;
     const int tiles = bwd_kv_tc5_tiles(t);
+    if (pair0 == 0) {
+        key_tile_plan_kernel<<<(tiles * 2 + 127) / 128, 128, 0, p.stream>>>(t, n_left, n_right, ranges, plan, tiles);
+        trace_mark(p.stream, "key_tile_plan");
+    }
     kernel<<<dim3(n_pairs, tiles), kKvThreads, BwdKvSmem::bytes, p.stream>>>(
-        t, n_left, n_right, p.lse, delta, aff_slab, (__nv_bfloat16*)p.dk, (__nv_bfloat16*)p.dv, drel_part, p.status,
+        t, n_left, n_right, ranges, plan, p.lse, delta, aff_slab, (__nv_bfloat16*)p.dk, (__nv_bfloat16*)p.dv, drel_part, p.status,
         p.H, pair0, p.scale, p.lengths, p.drop, tm_q, tm_g, tm_k, tm_v, tm_r);
     trace_mark(p.stream, "bwd_kv_tc5");
     const int n_rel = p.g->dims.n_rel, n_lv = max(n_left, n_right);

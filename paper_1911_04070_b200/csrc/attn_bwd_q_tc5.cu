@@ -139,9 +139,33 @@ __device__ __forceinline__ void q_rows_item(const RowCtx& rc, const uint32_t (&s
     }
 }
 
+// ranges[c * n + i] = (first, last) node of chunk c (left levels, then right levels) that token i attends, with the
+// conventions of fill_row_bounds and the self loop folded into the left range of level 0.  Both tensor-memory
+// backward kernels read the table instead of walking the levels again for every tile they visit.
+__global__ void level_ranges_kernel(TreeParams t, int n_left, int n_right, int2* __restrict__ ranges) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= t.n) return;
+    {
+        LeftWalk w(t, i);
+        for (int c = 0; c < n_left; ++c) {
+            int2 v = make_int2(0, -1);
+            if (w.valid()) { v = make_int2(w.lo, w.hi); w.next(); }
+            if (c == 0) v = v.x > v.y ? make_int2(i, i) : make_int2(v.x, i);
+            ranges[(size_t)c * t.n + i] = v;
+        }
+    }
+    RightWalk w(t, i);
+    for (int c = 0; c < n_right; ++c) {
+        const int n_l = t.n >> c;
+        int2 v = make_int2(n_l, n_l - 1);
+        if (w.valid()) { v = make_int2(w.lo, w.hi); w.next(); }
+        ranges[(size_t)(n_left + c) * t.n + i] = v;
+    }
+}
+
 template <bool kDrop>
 __global__ void __launch_bounds__(kQThreads, 1)
-bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
+bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__ ranges,
                  const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ out,
                  const float* __restrict__ lse, const __nv_bfloat16* __restrict__ d_out,
                  __nv_bfloat16* __restrict__ dq, float* __restrict__ delta_out, int* __restrict__ status,
@@ -193,13 +217,9 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right,
     }
     cp_async_commit();
     int2* bnd_abs = reinterpret_cast<int2*>(sk_s);  // absolute ranges, only until the relative table is written
-    if (tid < kQTok) {
-        fill_row_bounds<kQTok>(t, t0, tid, n_left, n_right, bnd_abs);
-        const int i = t0 + tid;  // the self loop joins the level-0 left range: it ends at the token itself
-        const int2 v0 = bnd_abs[tid];
-        bnd_abs[tid] = v0.x > v0.y ? make_int2(i, i) : make_int2(v0.x, i);
-        lse_s[tid] = lse[((size_t)b * N_nodes + i) * H + h] * kLog2e;
-    }
+    for (int idx = tid; idx < chunks * kQTok; idx += kQThreads)   // the rows' ranges, self loop included, from the table
+        bnd_abs[idx] = __ldg(ranges + (size_t)(idx / kQTok) * t.n + t0 + (idx % kQTok));
+    if (tid < kQTok) lse_s[tid] = lse[((size_t)b * N_nodes + t0 + tid) * H + h] * kLog2e;
     if (tid == 0) {
         tc5::mbar_init(bar(kBarSFull), 1);
         tc5::mbar_init(bar(kBarSFree), kQRowThreads);
@@ -516,8 +536,9 @@ bool bwd_q_tc5_fits(const TreeParams& t) {
     return n_items <= kQMaxItems && BwdQSmem::bytes(n_left + n_right) <= 227 * 1024;
 }
 
-// dq of the token rows, and the row terms d_out . out of the tokens into `delta` ([B * H][n] fp32).
-bpt_status launch_bwd_q_tc5(const AttnProblem& p, float* delta) {
+// dq of the token rows, the row terms d_out . out of the tokens into `delta` ([B * H][n] fp32) and the table of the
+// tokens' node ranges into `ranges` ([chunks][n] int2), which the key-side kernel reads too.
+bpt_status launch_bwd_q_tc5(const AttnProblem& p, float* delta, int2* ranges) {
     int n_left, n_right;
     context_levels(p.tree, &n_left, &n_right);
     const size_t smem = BwdQSmem::bytes(n_left + n_right);
@@ -529,8 +550,10 @@ bpt_status launch_bwd_q_tc5(const AttnProblem& p, float* delta) {
     if (!tc5::encode_tiled() || !tc5::node_rows_map(&tm_k, p.k, p.B, N, p.H) || !tc5::node_rows_map(&tm_v, p.v, p.B, N, p.H) ||
         !tc5::rel_rows_map(&tm_r, p.rel_emb, p.g->dims.n_rel))
         return BPT_ERR_CUDA;
+    level_ranges_kernel<<<(p.tree.n + 127) / 128, 128, 0, p.stream>>>(p.tree, n_left, n_right, ranges);
+    trace_mark(p.stream, "level_ranges");
     const dim3 grid(p.tree.n / kQTok, p.H, p.B);
-    kernel<<<grid, kQThreads, smem, p.stream>>>(p.tree, n_left, n_right, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.out,
+    kernel<<<grid, kQThreads, smem, p.stream>>>(p.tree, n_left, n_right, ranges, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.out,
                                                 p.lse, (const __nv_bfloat16*)p.d_out, (__nv_bfloat16*)p.dq, delta, p.status,
                                                 p.H, p.scale, p.lengths, p.drop, tm_k, tm_v, tm_r);
     trace_mark(p.stream, "bwd_q_tc5");

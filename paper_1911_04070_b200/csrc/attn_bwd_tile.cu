@@ -696,14 +696,17 @@ size_t pairs_for_budget(const TreeParams& t, const ChunkPlan& plan, int B, int H
 // ---- tensor-memory path (attn_bwd_q_tc5.cu, attn_bwd_kv_tc5.cu): no partial rows; its workspace holds the row
 // terms of all pairs and, per pass, the span pass's blocks and the d_rel partials ----
 bool bwd_q_tc5_fits(const TreeParams& t);
-bpt_status launch_bwd_q_tc5(const AttnProblem& p, float* delta);
+bpt_status launch_bwd_q_tc5(const AttnProblem& p, float* delta, int2* ranges);
 size_t bwd_kv_tc5_drel_floats(const TreeParams& t, int n_pairs);
-bpt_status launch_bwd_kv_tc5(const AttnProblem& p, int pair0, int n_pairs, const float* delta, const float* aff_slab, float* drel_part);
+int bwd_kv_tc5_tiles(const TreeParams& t);
+bpt_status launch_bwd_kv_tc5(const AttnProblem& p, int pair0, int n_pairs, const float* delta, const int2* ranges, int2* plan,
+                             const float* aff_slab, float* drel_part);
 
 namespace {
 
 struct Tc5Workspace {
     float *delta, *aff_slab, *ext_dq, *drel_part;
+    int2 *ranges, *plan;   // per token and chunk the node range; per key tile and side the query blocks
     int pairs_per_pass;
     size_t bytes;
 };
@@ -714,6 +717,10 @@ Tc5Workspace carve_tc5(const TreeParams& t, int B, int H, size_t pairs, void* ba
     char* c = (char*)base;
     size_t off = 0;
     w.delta = (float*)(c + off); off += align256(sizeof(float) * (size_t)B * H * t.n);
+    int n_left, n_right;
+    context_levels(t, &n_left, &n_right);
+    w.ranges = (int2*)(c + off); off += align256(sizeof(int2) * (size_t)(n_left + n_right) * t.n);
+    w.plan = (int2*)(c + off); off += align256(sizeof(int2) * (size_t)bwd_kv_tc5_tiles(t) * 2);
     w.aff_slab = (float*)(c + off); off += align256(sizeof(float) * bwd_span_slab_floats(t, (int)pairs));
     w.ext_dq = (float*)(c + off); off += align256(sizeof(float) * bwd_span_ext_floats(t, (int)pairs));
     w.drel_part = (float*)(c + off); off += align256(sizeof(float) * bwd_kv_tc5_drel_floats(t, (int)pairs));
@@ -734,19 +741,19 @@ size_t tc5_pairs_for_budget(const TreeParams& t, int B, int H, size_t budget) {
 // enough nodes per token; bpt_attn_options.path forces either family.
 bool want_bwd_tc5(const TreeParams& t, uint32_t path) {
     if (path == BPT_PATH_MMA || !bwd_q_tc5_fits(t)) return false;
-    return path == BPT_PATH_TC5 || t.k >= 32;
+    return path == BPT_PATH_TC5 || t.k >= 56;   // measured at n = 1024 .. 65536: ahead of the warp-level kernels at k = 64, level at k = 48
 }
 
 bpt_status launch_bwd_tc5(const AttnProblem& p) {
     const TreeParams& t = p.tree;
     const Tc5Workspace ws = carve_tc5(t, p.B, p.H, tc5_pairs_for_budget(t, p.B, p.H, p.workspace_bytes), p.workspace);
     if (ws.bytes > p.workspace_bytes) return BPT_ERR_WORKSPACE;
-    bpt_status s = launch_bwd_q_tc5(p, ws.delta);  // token dq and the row terms of every pair
+    bpt_status s = launch_bwd_q_tc5(p, ws.delta, ws.ranges);  // token dq, the row terms of every pair, the table of ranges
     const int total = p.B * p.H;
     for (int pair0 = 0; pair0 < total && s == BPT_OK; pair0 += ws.pairs_per_pass) {
         const int np = min(ws.pairs_per_pass, total - pair0);
         s = launch_bwd_span(p, pair0, np, ws.ext_dq, ws.aff_slab);  // span dq; per token the affiliated edges' share of dk / dv
-        if (s == BPT_OK) s = launch_bwd_kv_tc5(p, pair0, np, ws.delta, ws.aff_slab, ws.drel_part);
+        if (s == BPT_OK) s = launch_bwd_kv_tc5(p, pair0, np, ws.delta, ws.ranges, ws.plan, ws.aff_slab, ws.drel_part);
     }
     return s;
 }
