@@ -97,7 +97,8 @@ struct RowCtx {
 template <int kDir, bool kDrop>
 __device__ __forceinline__ void q_rows_item(const RowCtx& rc, const uint32_t (&sv)[kQPieces][kQCols], const uint32_t (&dv)[kQPieces][kQCols],
                                             int npieces, int ob, int omin, int orange, int ch0, int n_ch,
-                                            const DropoutParams& drop, uint32_t src0) {
+                                            const DropoutParams& drop, uint32_t src0,
+                                            uint32_t tiles_free_bar, uint32_t tiles_free_parity, bool must_wait, volatile int* abort_s) {
     const int r7 = rc.row & 7;
     const float* bp = rc.bias_row + ob * kQTok;
     // Per piece two phases, so that no shared-memory store stands between the table loads of its elements (the
@@ -118,6 +119,7 @@ __device__ __forceinline__ void q_rows_item(const RowCtx& rc, const uint32_t (&s
                 dsv[x] = in ? pr * (dp - rc.delta) : 0.f;
                 inm |= in ? 1u << x : 0u;
             }
+            if (p == 0 && must_wait && !*abort_s && !tc5::mbar_wait_fast(tiles_free_bar, tiles_free_parity)) *abort_s = 1;  // first store of the item: the dS tiles must be free
             // by-offset stores: the 8 offsets of this piece lie in at most two 16-byte chunks of the row
             const int of = ob + kDir * (p * 32);          // offset of the thread's first column of the piece
             const int a = of & 7, c1 = of >> 3, c2 = c1 + kDir;
@@ -446,8 +448,13 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__
             tc5::fence_before_sync();
             tc5::mbar_arrive(bar(kBarSFree));  // this thread holds its part: the next item's products may overwrite it
 
+            // The dS tiles are free once the products of the item before are done.  A chunk's first item needs that
+            // at once (it clears the by-offset tile; and since those products only started when every row thread had
+            // finished that item, nobody still reads the old bias values either); any other item only before its
+            // first store, so its wait hides behind the first piece's arithmetic.
+            const bool wait_late = j > 0 && !first && npieces > 0;
+            if (j > 0 && !wait_late) wait(kBarDsFree, (j - 1) & 1);
             if (first) {
-                quad_bar(quad);  // every thread of the row group is done with the previous chunk's bias values
                 // table entry = scale * log2(e) * q.r - lse * log2(e): the exponent of an edge is one fused multiply-add away
                 if (have_qr) {
 #pragma unroll
@@ -459,7 +466,6 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__
                     for (int x = 0; x < kQBiasRows - 64; ++x) bias_s[(64 + x) * kQTok + row] = fmaf(__uint_as_float(qr2[x]), scale_log2e, -rc.lse);
                 }
             }
-            if (j > 0) wait(kBarDsFree, (j - 1) & 1);  // the products that read the dS tiles of the item before are done
             if (first) {
                 // this row's entries of the by-offset tile start from zero (the row's four threads share the ten chunks)
                 for (int ch = part; ch < kQRelRows / 8; ch += kQTpr)
@@ -479,8 +485,8 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__
             const int orange = max(omax1 - omin, 0);
             uint32_t src0 = 0;
             if constexpr (kDrop) src0 = (uint32_t)(node_id(t.n, side ? it.c - n_left : it.c, 0) + crange[it.c].x + e0);
-            if (side) q_rows_item<1, kDrop>(rc, sv, dv, npieces, ob, omin, orange, ch0, n_ch, drop, src0);
-            else q_rows_item<-1, kDrop>(rc, sv, dv, npieces, ob, omin, orange, ch0, n_ch, drop, src0);
+            if (side) q_rows_item<1, kDrop>(rc, sv, dv, npieces, ob, omin, orange, ch0, n_ch, drop, src0, bar(kBarDsFree), (j - 1) & 1, wait_late, abort_s);
+            else q_rows_item<-1, kDrop>(rc, sv, dv, npieces, ob, omin, orange, ch0, n_ch, drop, src0, bar(kBarDsFree), (j - 1) & 1, wait_late, abort_s);
             for (int ci = part; ci < n_ch; ci += kQTpr)  // the rest of the row is zero
                 if (ci < ch0 || ci >= ch0 + npieces * 4)
                     *reinterpret_cast<uint4*>(ds_s + (ci >> 3) * (kQTok * 128) + tile_off(row, ci & 7)) = make_uint4(0, 0, 0, 0);
