@@ -39,6 +39,10 @@ constexpr int kKvTpr = 4;                        // threads per key row
 constexpr int kKvRowThreads = kKvKeys * kKvTpr;  // 16 warps
 constexpr int kKvThreads = kKvRowThreads + 96;   // + load warp + two MMA warps
 constexpr int kKvCols = kKvQB / kKvTpr;          // query columns per thread and item
+constexpr int kKvGrp = 16;                       // ... worked through in groups of 16 (one 16-column tensor-memory load)
+constexpr int kKvGroups = kKvCols / kKvGrp;
+constexpr int kKvChan = 64 / kKvTpr;             // output channels per thread in the read-out
+static_assert(kKvCols % kKvGrp == 0 && kKvChan % 16 == 0, "threads per key row: 1, 2 or 4");
 constexpr int kKvRing = 3;
 constexpr int kKvRelRows = 80;                   // relation rows per side (k + 2 <= 66), in 16-row boxes
 constexpr int kKvBiasStride = 66;
@@ -107,26 +111,27 @@ __global__ void key_tile_plan_kernel(TreeParams t, int n_left, int n_right, cons
     plan[id] = out;
 }
 
-// One item's share of a row thread: its key node m against kKvCols query columns.  Predicated, no branch per element.
+// One group of an item's share of a row thread: its key node m against kKvGrp query columns (col0 .. col0 + 15 of the
+// block).  Predicated, no branch per element.
 // kSide: 1 = the keys are right context of the queries (offset m - lo), 0 = left context (offset hi - m).
 // Two phases, so that no shared-memory store stands between the loads of different elements (the compiler must
 // assume the by-offset stores alias the tables): first every weight, then every store.  The by-offset store of a
 // missing edge goes, with value zero, to row 127 of the tile, which is no relation offset.
 template <int kSide, bool kDrop>
-__device__ __forceinline__ void kv_rows_item(const uint32_t (&sv)[kKvCols], const uint32_t (&dv)[kKvCols], const QMeta* __restrict__ mq,
-                                             const float* __restrict__ bias_col, unsigned char* __restrict__ skw, int m, int part,
+__device__ __forceinline__ void kv_rows_item(const uint32_t* __restrict__ sv, const uint32_t* __restrict__ dv, const QMeta* __restrict__ mq,
+                                             const float* __restrict__ bias_col, unsigned char* __restrict__ skw, int m, int col0,
                                              float scale_log2e, const DropoutParams& drop, uint32_t pair, uint32_t dst0, uint32_t src,
-                                             uint32_t (&pp)[kKvCols / 2], uint32_t (&dd)[kKvCols / 2]) {
-    uint32_t at[kKvCols];  // byte offset of each element's by-offset store
+                                             uint32_t* __restrict__ pp, uint32_t* __restrict__ dd) {
+    uint32_t at[kKvGrp];  // byte offset of each element's by-offset store
 #pragma unroll
-    for (int x = 0; x < kKvCols; x += 2) {
+    for (int x = 0; x < kKvGrp; x += 2) {
         float pv[2], dsv[2];
 #pragma unroll
         for (int y = 0; y < 2; ++y) {
             const QMeta a = mq[x + y];
             const bool in = m >= a.lo && m <= a.hi;
             const int off = kSide ? m - a.lo : a.hi - m;
-            const int col = part * kKvCols + x + y;
+            const int col = col0 + x + y;
             const float bias = in ? bias_col[(x + y) * kKvBiasStride + off] : 0.f;
             float pr = ex2f(fmaf(__uint_as_float(sv[x + y]), scale_log2e, bias));
             float dp = __uint_as_float(dv[x + y]), d;
@@ -146,7 +151,7 @@ __device__ __forceinline__ void kv_rows_item(const uint32_t (&sv)[kKvCols], cons
         dd[x >> 1] = pack_bf16(dsv[0], dsv[1]);
     }
 #pragma unroll
-    for (int x = 0; x < kKvCols; ++x)
+    for (int x = 0; x < kKvGrp; ++x)
         *reinterpret_cast<uint16_t*>(skw + at[x]) = (uint16_t)((x & 1) ? dd[x >> 1] >> 16 : dd[x >> 1] & 0xffffu);
 }
 
@@ -349,9 +354,13 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict_
             wait(kvSFull, j & 1);
             tc5::fence_after_sync();
             uint32_t sv[kKvCols], dv[kKvCols], qr[kKvCols];
-            tc5::tmem_ld16(tbase + lane_base + kKvColS + part * kKvCols, sv);
-            tc5::tmem_ld16(tbase + lane_base + kKvColDP + part * kKvCols, dv);
-            if (quad < 3) tc5::tmem_ld16(tbase + lane_base + kKvColQR + part * kKvCols, qr);  // lanes = relation offsets here
+#pragma unroll
+            for (int gq = 0; gq < kKvGroups; ++gq) {
+                tc5::tmem_ld16(tbase + lane_base + kKvColS + part * kKvCols + gq * kKvGrp, *reinterpret_cast<uint32_t (*)[16]>(sv + gq * kKvGrp));
+                tc5::tmem_ld16(tbase + lane_base + kKvColDP + part * kKvCols + gq * kKvGrp, *reinterpret_cast<uint32_t (*)[16]>(dv + gq * kKvGrp));
+                if (quad < 3)   // lanes = relation offsets here
+                    tc5::tmem_ld16(tbase + lane_base + kKvColQR + part * kKvCols + gq * kKvGrp, *reinterpret_cast<uint32_t (*)[16]>(qr + gq * kKvGrp));
+            }
             tc5::tmem_ld_wait();
             tc5::fence_before_sync();
             tc5::mbar_arrive(bar(kvSFree));
@@ -369,14 +378,21 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict_
             // does any of the warp's 32 keys meet any of this thread group's 16 queries?
             bool hit = false;
             if (lane < kKvCols) { const QMeta a = mq[lane]; hit = a.lo <= a.hi && a.hi >= mw0 && a.lo <= mw0 + 31; }
+            const unsigned hits = __ballot_sync(0xffffffffu, hit);
             uint32_t pp[kKvCols / 2], dd[kKvCols / 2];
 #pragma unroll
             for (int x = 0; x < kKvCols / 2; ++x) pp[x] = dd[x] = 0u;
-            if (__any_sync(0xffffffffu, hit)) {
-                const float* bias_col = bias + part * kKvCols * kKvBiasStride;
-                const uint32_t src = (uint32_t)(id0 + m), dst0 = (uint32_t)(q0 + part * kKvCols);
-                if (side) kv_rows_item<1, kDrop>(sv, dv, mq, bias_col, skw, m, part, scale_log2e, drop, (uint32_t)pair, dst0, src, pp, dd);
-                else kv_rows_item<0, kDrop>(sv, dv, mq, bias_col, skw, m, part, scale_log2e, drop, (uint32_t)pair, dst0, src, pp, dd);
+#pragma unroll
+            for (int gq = 0; gq < kKvGroups; ++gq) {
+                if ((hits >> (gq * kKvGrp)) & 0xffffu) {   // some of the warp's keys meet some of the group's queries
+                    const int col0 = part * kKvCols + gq * kKvGrp;
+                    const float* bias_col = bias + col0 * kKvBiasStride;
+                    const uint32_t src = (uint32_t)(id0 + m), dst0 = (uint32_t)(q0 + col0);
+                    if (side) kv_rows_item<1, kDrop>(sv + gq * kKvGrp, dv + gq * kKvGrp, mq + gq * kKvGrp, bias_col, skw, m, col0, scale_log2e, drop,
+                                                     (uint32_t)pair, dst0, src, pp + gq * (kKvGrp / 2), dd + gq * (kKvGrp / 2));
+                    else kv_rows_item<0, kDrop>(sv + gq * kKvGrp, dv + gq * kKvGrp, mq + gq * kKvGrp, bias_col, skw, m, col0, scale_log2e, drop,
+                                                (uint32_t)pair, dst0, src, pp + gq * (kKvGrp / 2), dd + gq * (kKvGrp / 2));
+                }
             }
             if (j > 0) wait(kvDsFree, (j - 1) & 1);   // the products that read P^T, dS^T of the item before are done (hidden behind the weights above)
 #pragma unroll
@@ -397,55 +413,63 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict_
         // ---- results: dk, dv rows (plus, for tokens, what the span rows left for them), d_rel partials ----
         if (J > 0) wait(kvDsFree, (J - 1) & 1);
         tc5::fence_after_sync();
-        uint32_t xk[16], xv[16];
-        if (J > 0) {
-            tc5::tmem_ld16(tbase + lane_base + kKvColDK + part * 16, xk);
-            tc5::tmem_ld16(tbase + lane_base + kKvColDV + part * 16, xv);
-            tc5::tmem_ld_wait();
-        } else {
 #pragma unroll
-            for (int x = 0; x < 16; ++x) xk[x] = xv[x] = 0u;
-        }
-        if (level == 0 && m < t.n) {  // affiliated edges: the span pass's share of this token's dk / dv
-            const float4* a = reinterpret_cast<const float4*>(aff_slab + ((size_t)pl * t.n + m) * 128 + part * 16);
+        for (int cg = 0; cg < kKvChan / 16; ++cg) {   // this thread's output channels, sixteen at a time
+            const int ch0 = part * kKvChan + cg * 16;
+            uint32_t xk[16], xv[16];
+            if (J > 0) {
+                tc5::tmem_ld16(tbase + lane_base + kKvColDK + ch0, xk);
+                tc5::tmem_ld16(tbase + lane_base + kKvColDV + ch0, xv);
+                tc5::tmem_ld_wait();
+            } else {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const float4 ak = __ldg(a + c), av = __ldg(a + 16 + c);
-                xk[4 * c] = __float_as_uint(__uint_as_float(xk[4 * c]) + ak.x); xk[4 * c + 1] = __float_as_uint(__uint_as_float(xk[4 * c + 1]) + ak.y);
-                xk[4 * c + 2] = __float_as_uint(__uint_as_float(xk[4 * c + 2]) + ak.z); xk[4 * c + 3] = __float_as_uint(__uint_as_float(xk[4 * c + 3]) + ak.w);
-                xv[4 * c] = __float_as_uint(__uint_as_float(xv[4 * c]) + av.x); xv[4 * c + 1] = __float_as_uint(__uint_as_float(xv[4 * c + 1]) + av.y);
-                xv[4 * c + 2] = __float_as_uint(__uint_as_float(xv[4 * c + 2]) + av.z); xv[4 * c + 3] = __float_as_uint(__uint_as_float(xv[4 * c + 3]) + av.w);
+                for (int x = 0; x < 16; ++x) xk[x] = xv[x] = 0u;
             }
-        }
+            if (level == 0 && m < t.n) {  // affiliated edges: the span pass's share of this token's dk / dv
+                const float4* a = reinterpret_cast<const float4*>(aff_slab + ((size_t)pl * t.n + m) * 128 + ch0);
 #pragma unroll
-        for (int c = 0; c < 2; ++c) {  // rounded once; staged in the K / V tiles for coalesced stores
-            uint32_t a[4], bq[4];
-#pragma unroll
-            for (int y = 0; y < 4; ++y) {
-                a[y] = pack_bf16(__uint_as_float(xk[c * 8 + 2 * y]) * scale, __uint_as_float(xk[c * 8 + 2 * y + 1]) * scale);
-                bq[y] = pack_bf16(__uint_as_float(xv[c * 8 + 2 * y]), __uint_as_float(xv[c * 8 + 2 * y + 1]));
+                for (int c = 0; c < 4; ++c) {
+                    const float4 ak = __ldg(a + c), av = __ldg(a + 16 + c);
+                    xk[4 * c] = __float_as_uint(__uint_as_float(xk[4 * c]) + ak.x); xk[4 * c + 1] = __float_as_uint(__uint_as_float(xk[4 * c + 1]) + ak.y);
+                    xk[4 * c + 2] = __float_as_uint(__uint_as_float(xk[4 * c + 2]) + ak.z); xk[4 * c + 3] = __float_as_uint(__uint_as_float(xk[4 * c + 3]) + ak.w);
+                    xv[4 * c] = __float_as_uint(__uint_as_float(xv[4 * c]) + av.x); xv[4 * c + 1] = __float_as_uint(__uint_as_float(xv[4 * c + 1]) + av.y);
+                    xv[4 * c + 2] = __float_as_uint(__uint_as_float(xv[4 * c + 2]) + av.z); xv[4 * c + 3] = __float_as_uint(__uint_as_float(xv[4 * c + 3]) + av.w);
+                }
             }
-            *reinterpret_cast<uint4*>(k_s + tile_off(row, part * 2 + c)) = make_uint4(a[0], a[1], a[2], a[3]);
-            *reinterpret_cast<uint4*>(v_s + tile_off(row, part * 2 + c)) = make_uint4(bq[0], bq[1], bq[2], bq[3]);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {  // rounded once; staged in the K / V tiles for coalesced stores
+                uint32_t a[4], bq[4];
+#pragma unroll
+                for (int y = 0; y < 4; ++y) {
+                    a[y] = pack_bf16(__uint_as_float(xk[c * 8 + 2 * y]) * scale, __uint_as_float(xk[c * 8 + 2 * y + 1]) * scale);
+                    bq[y] = pack_bf16(__uint_as_float(xv[c * 8 + 2 * y]), __uint_as_float(xv[c * 8 + 2 * y + 1]));
+                }
+                *reinterpret_cast<uint4*>(k_s + tile_off(row, (ch0 >> 3) + c)) = make_uint4(a[0], a[1], a[2], a[3]);
+                *reinterpret_cast<uint4*>(v_s + tile_off(row, (ch0 >> 3) + c)) = make_uint4(bq[0], bq[1], bq[2], bq[3]);
+            }
         }
         // d_rel partials of this CTA: [side][offset][channel], zero where the side brought nothing
         if (quad < 3) {  // lanes = relation offsets; the loads are warp-wide, the stores take the offsets in use
 #pragma unroll
             for (int s = 0; s < 2; ++s) {
                 if (!side_on[s]) continue;
-                uint32_t xr[16];
-                if (nb_side[s] > 0) {
-                    tc5::tmem_ld16(tbase + lane_base + kKvColDR + s * 64 + part * 16, xr);
-                    tc5::tmem_ld_wait();
-                } else {
 #pragma unroll
-                    for (int x = 0; x < 16; ++x) xr[x] = 0u;
+                for (int cg = 0; cg < kKvChan / 16; ++cg) {
+                    const int ch0 = part * kKvChan + cg * 16;
+                    uint32_t xr[16];
+                    if (nb_side[s] > 0) {
+                        tc5::tmem_ld16(tbase + lane_base + kKvColDR + s * 64 + ch0, xr);
+                        tc5::tmem_ld_wait();
+                    } else {
+#pragma unroll
+                        for (int x = 0; x < 16; ++x) xr[x] = 0u;
+                    }
+                    if (row >= kKvBiasStride) continue;
+                    float4* dst = reinterpret_cast<float4*>(drel_part + ((((size_t)pl * gridDim.y + blockIdx.y) * 2 + s) * kKvBiasStride + row) * 64 + ch0);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        dst[c] = make_float4(__uint_as_float(xr[4 * c]), __uint_as_float(xr[4 * c + 1]), __uint_as_float(xr[4 * c + 2]), __uint_as_float(xr[4 * c + 3]));
                 }
-                if (row >= kKvBiasStride) continue;
-                float4* dst = reinterpret_cast<float4*>(drel_part + ((((size_t)pl * gridDim.y + blockIdx.y) * 2 + s) * kKvBiasStride + row) * 64 + part * 16);
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    dst[c] = make_float4(__uint_as_float(xr[4 * c]), __uint_as_float(xr[4 * c + 1]), __uint_as_float(xr[4 * c + 2]), __uint_as_float(xr[4 * c + 3]));
             }
         }
     }
