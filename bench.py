@@ -51,9 +51,9 @@ KERNEL_MODEL = {
 # were read; when the file has changed since, the bench reports traffic = null instead of a stale number.
 NCU_DRAM_BYTES_PER_PAIR = {
     # kernel: (bytes per pair, source file, sha256 of the file at capture time (first 16 hex digits))
-    "fwd_tc5": (41.28e6 / 8, "attn_fwd_tc5.cu", ""),
-    "bwd_q_tc5": (61.13e6 / 8, "attn_bwd_q_tc5.cu", ""),
-    "bwd_kv_tc5": (106.98e6 / 8, "attn_bwd_kv_tc5.cu", ""),
+    "fwd_tc5": (41.22e6 / 8, "attn_fwd_tc5.cu", "812e238b1a1e6f78"),
+    "bwd_q_tc5": (60.39e6 / 8, "attn_bwd_q_tc5.cu", "d3e9f827fddbbe6a"),
+    "bwd_kv_tc5": (118.41e6 / 8, "attn_bwd_kv_tc5.cu", "e39a0a104ddf814d"),
 }
 FLOPS_PER_EDGE_HEAD = {"fwd": 6, "bwd": 14}   # x d_head: q.k, q.r, P.v forward; s again, dP, dq, dk, dv, d_rel backward
 
