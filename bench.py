@@ -249,11 +249,13 @@ def run_ours(args, cfg_name, cfg):
     dq, dk, dv = (torch.empty_like(t["q"]) for _ in range(3))
     d_rel = torch.empty((g.n_rel, d), dtype=torch.float32, device=dev)
 
+    path = {"auto": binding.BPT_PATH_AUTO, "mma": binding.BPT_PATH_MMA, "tc5": binding.BPT_PATH_TC5}[args.path]
+
     def step():
-        binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out=out, lse=lse, workspace=ws)
+        binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out=out, lse=lse, workspace=ws, path=path)
         if do_bwd:
             binding.bpt_attn_bwd(g, t["q"], t["k"], t["v"], t["rel_emb"], scale, out, lse, t["d_out"], workspace=ws,
-                                 dq=dq, dk=dk, dv=dv, d_rel=d_rel)
+                                 dq=dq, dk=dk, dv=dv, d_rel=d_rel, path=path)
             shard.allreduce_d_rel(d_rel)
 
     def barrier():
@@ -311,6 +313,9 @@ def run_ours(args, cfg_name, cfg):
             marks += binding.bpt_trace_end(16)
         barrier()
     t_end = time.time()
+    device_status = binding.bpt_check(ws)   # a bounded device-side wait that ran out would make the timed results invalid
+    if device_status:
+        raise SystemExit("device-side failure report: %s" % binding.status_str(device_status))
     ms_total = max_over_ranks(ms_sum)
     clocks = sampler.stop(t_begin, t_end) if rank == 0 else None
     ms_step = ms_total / args.steps
@@ -345,10 +350,10 @@ def run_ours(args, cfg_name, cfg):
         s_comp.wait_event(in_ready[buf])
         if i >= 2:
             s_comp.wait_event(out_copied[buf])         # this result set has been read out
-        binding.bpt_attn_fwd(g, ti["q"], ti["k"], ti["v"], ti["rel_emb"], scale, out=rd[0], lse=rd[1], workspace=ws)
+        binding.bpt_attn_fwd(g, ti["q"], ti["k"], ti["v"], ti["rel_emb"], scale, out=rd[0], lse=rd[1], workspace=ws, path=path)
         if do_bwd:
             binding.bpt_attn_bwd(g, ti["q"], ti["k"], ti["v"], ti["rel_emb"], scale, rd[0], rd[1], ti["d_out"], workspace=ws,
-                                 dq=rd[2], dk=rd[3], dv=rd[4], d_rel=rd[5])
+                                 dq=rd[2], dk=rd[3], dv=rd[4], d_rel=rd[5], path=path)
             shard.allreduce_d_rel(rd[5])
         comp_done[buf].record(s_comp)
         with torch.cuda.stream(s_out):
@@ -430,7 +435,8 @@ def run_ours(args, cfg_name, cfg):
         "config": {"workload": cfg_name, "n": cfg["n"], "k": cfg["k"], "left_only": bool(cfg["flags"] & 1),
                    "batch_per_gpu": B, "heads": H, "d_head": d, "edges_per_sequence": E,
                    "pass": "fwd+bwd" if do_bwd else "fwd",
-                   "l2": "flushed by a 256 MB write between timed steps" if flush else "inputs larger than L2", "parallelism": "batch shards x%d" % world},
+                   "l2": "flushed by a 256 MB write between timed steps" if flush else "inputs larger than L2", "parallelism": "batch shards x%d" % world,
+                   "kernels": args.path},
         "edge_heads_per_s": value * H, "tokens_per_s": world * B * cfg["n"] / (ms_step * 1e-3),
         "hbm_roofline_frac_step": step_roof_ms / ms_step, "hbm_roofline_ms_step": step_roof_ms,
         "compulsory_hbm_ms_step": compulsory_ms, "compulsory_hbm_frac_step": compulsory_ms / ms_step,
@@ -558,6 +564,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="cfg4_char_lm")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--path", default="auto", choices=["auto", "mma", "tc5"],
+                    help="kernel family of the token rows: the library's choice by k, the warp-level (mma.sync) kernels, or the tensor-memory (tcgen05) kernels")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (profiling of a smaller case)")
     ap.add_argument("--sweep", action="store_true", help="run the n x k scaling sweep instead: one JSON line per point")
     ap.add_argument("--model", action="store_true", help="time a 6-layer BPT stack (Sec. 4.4 setting) instead: one JSON line per point")
