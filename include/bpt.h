@@ -244,6 +244,22 @@ bpt_status bpt_attn_fwd_rows(const bpt_graph* g, int32_t B, int32_t H, int32_t d
                              void* out, float* lse, void* cuda_stream);
 
 /*
+ * Output projection, residual and layer normalisation of a layer in one kernel (Algorithm 2 of Sec. 3.3:
+ * Z = norm(H + GSA(H) W^O), with the output projection W^O of Sec. 3.1):
+ *     z[r, :] = LayerNorm(h[r, :] + a[r, :] w_o^T) * gamma + beta        for every row r,
+ * where a is the attention output with the heads concatenated ([B, n_nodes, H, d] seen as [rows, D], D = H * d),
+ * w_o is [D, D] with row o holding the weights of output channel o (the layout of a linear layer's weight),
+ * h the layer's input states [rows, D], gamma / beta the normalisation's scale and shift [D] (fp32), z the
+ * result [rows, D].  a, w_o, h, z are bf16, contiguous and 16-byte aligned; the product accumulates in fp32 and
+ * mean / variance (biased, about the mean) are taken in fp32 over the D channels; one rounding to bf16.
+ * D must be 128, 256 or 512; rows >= 1.  `workspace` is NULL or a device buffer of at least 256 bytes that
+ * receives the status block (see bpt_check).  Forward only: training goes through the separate operators.
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+bpt_status bpt_out_proj_norm(const void* a, const void* w_o, const void* h, const float* gamma, const float* beta,
+                             void* z, int64_t rows, int32_t D, float eps, void* workspace, void* cuda_stream);
+
+/*
  * Backward pass for callers that must not allocate device memory (the paper has no
  * counterpart; this is a deployment convenience).
  *

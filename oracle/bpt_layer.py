@@ -48,6 +48,15 @@ def attention(q, k, v, r, mask, rel, scale):
     return torch.einsum("bhuv,bvhc->buhc", p, v)
 
 
+def out_proj_norm(a, w_o, h, gamma, beta, eps=1e-5):
+    """The middle of Algorithm 2 written out in NumPy float64: z = LayerNorm(h + a w_o^T) * gamma + beta over the
+    last axis, with the biased variance about the mean (the definition of layer normalisation)."""
+    x = np.asarray(h, dtype=np.float64) + np.asarray(a, dtype=np.float64) @ np.asarray(w_o, dtype=np.float64).T
+    mean = x.mean(axis=-1, keepdims=True)
+    var = ((x - mean) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mean) / np.sqrt(var + eps) * np.asarray(gamma, dtype=np.float64) + np.asarray(beta, dtype=np.float64)
+
+
 def layer_forward(h, w, mask, rel, n_heads):
     """h: [B, N, D]; w: dict of float64 tensors wq, wk, wv, wo [D, D] (applied as x @ w.T), rel_emb [n_rel, D/H],
     ln1_w, ln1_b, ln2_w, ln2_b [D], ff1_w [F, D], ff1_b [F], ff2_w [D, F], ff2_b [D]."""

@@ -23,7 +23,7 @@ EXPORTS = ("bpt_graph_dims_query", "bpt_build_graph", "bpt_attn_workspace_bytes"
            "bpt_attn_bwd", "bpt_status_str", "bpt_trace_begin", "bpt_trace_end",
            "bpt_static_scratch_bytes", "bpt_attn_bwd_static_scratch", "bpt_attn_fwd_varlen", "bpt_attn_bwd_varlen",
            "bpt_attn_fwd_ex", "bpt_attn_bwd_ex", "bpt_attn_fwd_rows", "bpt_attn_bwd_min_workspace_bytes", "bpt_check",
-           "bpt_selftest_wait_timeout", "bpt_debug_bounds")
+           "bpt_selftest_wait_timeout", "bpt_debug_bounds", "bpt_out_proj_norm")
 
 
 class BptError(RuntimeError):
@@ -77,6 +77,8 @@ def load_library() -> ctypes.CDLL:
         lib.bpt_check.argtypes = [vp, vp]
         lib.bpt_selftest_wait_timeout.restype = ctypes.c_int
         lib.bpt_selftest_wait_timeout.argtypes = [vp, ctypes.c_int64, i32, vp]
+        lib.bpt_out_proj_norm.restype = ctypes.c_int
+        lib.bpt_out_proj_norm.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_int64, i32, f32, vp, vp]
         lib.bpt_debug_bounds.restype = ctypes.c_int
         lib.bpt_debug_bounds.argtypes = [ctypes.POINTER(ctypes.c_uint32), vp]
         lib.bpt_attn_fwd.restype = ctypes.c_int
@@ -198,6 +200,27 @@ def bpt_check(workspace) -> int:
     dev = torch.cuda.current_device() if workspace is None else workspace.device
     with torch.cuda.device(dev):
         return int(load_library().bpt_check(_ptr(workspace), _stream()))
+
+
+def bpt_out_proj_norm(a, w_o, h, gamma, beta, eps: float = 1e-5, z=None, workspace=None):
+    """z = LayerNorm(h + a @ w_o.T) * gamma + beta over the last axis, in one kernel (bf16 in and out, fp32
+    accumulation and statistics).  a, h: [..., D] bfloat16 contiguous; w_o: [D, D] bfloat16; gamma, beta: [D]
+    float32; D in (128, 256, 512).  Forward only."""
+    D = a.shape[-1]
+    for t in (a, h):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous() or t.shape != a.shape or not t.is_cuda:
+            raise ValueError("a and h must be contiguous bfloat16 CUDA tensors of one shape")
+    if w_o.dtype != torch.bfloat16 or w_o.shape != (D, D) or not w_o.is_contiguous():
+        raise ValueError("w_o must be a contiguous bfloat16 [D, D] tensor")
+    for t in (gamma, beta):
+        if t.dtype != torch.float32 or t.shape != (D,) or not t.is_contiguous():
+            raise ValueError("gamma and beta must be contiguous float32 [D] tensors")
+    rows = a.numel() // D
+    with torch.cuda.device(a.device):
+        z = torch.empty_like(a) if z is None else z
+        _check(load_library().bpt_out_proj_norm(_ptr(a), _ptr(w_o), _ptr(h), _ptr(gamma), _ptr(beta), _ptr(z), rows, D, float(eps),
+                                                _ptr(workspace), _stream()), "bpt_out_proj_norm")
+    return z
 
 
 def bpt_debug_bounds():

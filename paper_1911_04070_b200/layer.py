@@ -15,6 +15,11 @@ from torch import nn
 from . import binding
 
 
+# Inference (no gradient, bfloat16, model width 128 / 256 / 512): the output projection, the residual and the first
+# layer normalisation of a layer run in the library's fused kernel (bpt_out_proj_norm) instead of three operators.
+FUSE_OUT_PROJ_NORM = True
+
+
 class _GraphSelfAttention(torch.autograd.Function):
     """out = GSA(q, k, v, rel_emb) over the BPT graph; backward through bpt_attn_bwd."""
 
@@ -74,7 +79,12 @@ class BPTLayer(nn.Module):
         seed = int(torch.randint(0, 2 ** 62, (1,)).item()) if p_drop else 0   # a fresh mask per call, from torch's CPU generator
         a = graph_self_attention(self.g, split(self.wq(h)), split(self.wk(h)), split(self.wv(h)),
                                  self.rel_emb.to(h.dtype), lengths=lengths, dropout_p=p_drop, dropout_seed=seed)
-        z = self.norm1(h + self.wo(a.reshape(B, N, D)))
+        if (FUSE_OUT_PROJ_NORM and not torch.is_grad_enabled() and h.dtype == torch.bfloat16 and D in (128, 256, 512)
+                and self.wo.weight.dtype == torch.bfloat16):
+            z = binding.bpt_out_proj_norm(a.reshape(B, N, D), self.wo.weight.contiguous(), h.contiguous(), self.norm1.weight.float(),
+                                          self.norm1.bias.float(), self.norm1.eps)
+        else:
+            z = self.norm1(h + self.wo(a.reshape(B, N, D)))
         return self.norm2(z + self.ff2(torch.relu(self.ff1(z))))
 
 
