@@ -523,6 +523,10 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__
 
 }  // namespace
 
+void launch_level_ranges(const TreeParams& t, int n_left, int n_right, int2* ranges, cudaStream_t stream) {
+    level_ranges_kernel<<<(t.n + 127) / 128, 128, 0, stream>>>(t, n_left, n_right, ranges);
+}
+
 int bwd_q_tc5_chunks(const TreeParams& t) {
     int n_left, n_right;
     context_levels(t, &n_left, &n_right);
@@ -556,7 +560,7 @@ bpt_status launch_bwd_q_tc5(const AttnProblem& p, float* delta, int2* ranges) {
     if (!tc5::encode_tiled() || !tc5::node_rows_map(&tm_k, p.k, p.B, N, p.H) || !tc5::node_rows_map(&tm_v, p.v, p.B, N, p.H) ||
         !tc5::rel_rows_map(&tm_r, p.rel_emb, p.g->dims.n_rel))
         return BPT_ERR_CUDA;
-    level_ranges_kernel<<<(p.tree.n + 127) / 128, 128, 0, p.stream>>>(p.tree, n_left, n_right, ranges);
+    launch_level_ranges(p.tree, n_left, n_right, ranges, p.stream);
     trace_mark(p.stream, "level_ranges");
     const dim3 grid(p.tree.n / kQTok, p.H, p.B);
     kernel<<<grid, kQThreads, smem, p.stream>>>(p.tree, n_left, n_right, ranges, (const __nv_bfloat16*)p.q, (const __nv_bfloat16*)p.out,

@@ -157,7 +157,8 @@ static bpt_status launch_rows(const AttnProblem& p, int row0, int nrows, const i
 
 bpt_status launch_fwd_tile(const AttnProblem& p);
 bool fwd_tc5_eligible(const AttnProblem& p);
-bpt_status launch_fwd_tc5(const AttnProblem& p, int* status);
+bpt_status launch_fwd_tc5(const AttnProblem& p, int* status, int2* ranges);
+size_t fwd_tc5_ranges_bytes(const TreeParams& t);
 size_t fwd_span_workspace_bytes(const TreeParams& t, int B, int H);
 bpt_status launch_fwd_span(const AttnProblem& p);
 
@@ -167,7 +168,8 @@ size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dt
     if (!tile_path(g.dims.n, g.dims.k, d, dtype == BPT_BF16)) return 0;
     TreeParams t;
     tree_params_from_dims(g.dims, &t);
-    return span_ws_bytes(t, B, H) + 256;  // never empty, so that the status block in front of it exists for the tensor-memory kernel
+    // the span partials, then the node-range table of the tensor-memory kernel (never empty, so that the status block in front exists)
+    return span_ws_bytes(t, B, H) + fwd_tc5_ranges_bytes(t) + 256;
 }
 
 // Two kernels cover the token rows: the warp-level one (mma.sync, 64-token tiles) and the tensor-memory
@@ -179,7 +181,8 @@ static bool want_tc5(int k, uint32_t path) { return path == BPT_PATH_TC5 || (pat
 
 bpt_status launch_fwd(const AttnProblem& p) {
     if (tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16)) {  // token rows and span rows on the tensor cores
-        const bpt_status s = (want_tc5(p.tree.k, p.path) && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, p.status) : launch_fwd_tile(p);
+        int2* ranges = reinterpret_cast<int2*>(static_cast<char*>(p.workspace) + span_ws_bytes(p.tree, p.B, p.H));
+        const bpt_status s = (want_tc5(p.tree.k, p.path) && fwd_tc5_eligible(p)) ? launch_fwd_tc5(p, p.status, ranges) : launch_fwd_tile(p);
         return s != BPT_OK ? s : launch_fwd_span(p);
     }
     const int row0 = 0, nrows = p.g->dims.n_nodes;
