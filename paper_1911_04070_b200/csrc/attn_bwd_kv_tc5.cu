@@ -194,6 +194,10 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict_
         if (*abort_s) return;
         if (!tc5::mbar_wait_fast(bar(i), parity)) *abort_s = 1;
     };
+    auto wait_idle = [&](int i, uint32_t parity) {  // for the load and MMA threads: suspends instead of spinning
+        if (*abort_s) return;
+        if (!tc5::mbar_wait_idle(bar(i), parity)) *abort_s = 1;
+    };
     const int len = seq_len(lengths, b, t.n);
     const bool side_on[2] = {level < n_left, level < n_right};
 
@@ -250,7 +254,7 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict_
                 int side, q0;
                 item_of(j, side, q0);
                 const int rb = j % kKvRing, ru = j / kKvRing;
-                if (ru > 0) wait(kvQFree + rb, (ru - 1) & 1);
+                if (ru > 0) wait_idle(kvQFree + rb, (ru - 1) & 1);
                 if (lane == 0) {
                     tc5::mbar_expect_tx(bar(kvQFull + rb), 2u * (kKvQB / 16) * 2048u);
                     for (int x = 0; x < kKvQB / 16; ++x) {
@@ -294,9 +298,9 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict_
                 int side, q0;
                 item_of(j, side, q0);
                 const int rb = j % kKvRing, ru = j / kKvRing;
-                if (j == 0) wait(kvTiles, 0);
-                wait(kvQFull + rb, ru & 1);
-                if (j > 0) wait(kvSFree, (j - 1) & 1);
+                if (j == 0) wait_idle(kvTiles, 0);
+                wait_idle(kvQFull + rb, ru & 1);
+                if (j > 0) wait_idle(kvSFree, (j - 1) & 1);
                 if (*abort_s) break;
                 tc5::fence_after_sync();
                 const uint32_t q_lo = tc5::desc_lo_k_major(q_u + rb * (kKvQB * 128)), g_lo = tc5::desc_lo_k_major(g_u + rb * (kKvQB * 128)),
@@ -319,7 +323,7 @@ bwd_kv_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict_
                 int side, q0;
                 item_of(j, side, q0);
                 const int rb = j % kKvRing;
-                wait(kvDsFull, j & 1);
+                wait_idle(kvDsFull, j & 1);
                 if (*abort_s) break;
                 tc5::fence_after_sync();
                 const uint32_t q_lo = tc5::desc_lo_mn_major(q_u + rb * (kKvQB * 128)), g_lo = tc5::desc_lo_mn_major(g_u + rb * (kKvQB * 128));

@@ -207,6 +207,10 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__
         if (*abort_s) return;
         if (!tc5::mbar_wait_fast(bar(i), parity)) *abort_s = 1;
     };
+    auto wait_idle = [&](int i, uint32_t parity) {  // for the load and MMA threads: suspends instead of spinning
+        if (*abort_s) return;
+        if (!tc5::mbar_wait_idle(bar(i), parity)) *abort_s = 1;
+    };
 
     // ---- prologue: Q, d_out and out tiles, row terms, row ranges, barriers, tensor memory ----
     unsigned char* o_s = ds_s;  // the forward's output rows, only until the row terms are known
@@ -326,17 +330,17 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__
                 if (it.flags & 1) {
                     ++ci;
                     const int rb = ci & 1, ru = ci >> 1;
-                    if (ru > 0) wait(kBarRFree + rb, (ru - 1) & 1);
+                    if (ru > 0) wait_idle(kBarRFree + rb, (ru - 1) & 1);
                     const int rel_base = it.c == 0 ? 0 : (side ? rel_right(t, level, 0) : rel_left(t, level, 0));
                     tc5::mbar_expect_tx(bar(kBarRFull + rb), (uint32_t)(rel_cols / 16) * 2048u);
                     for (int x = 0; x < rel_cols / 16; ++x)
                         tc5::tma_load_2d(r_u + rb * (kQRelRows * 128) + x * 2048, &tm_r, 0, rel_base + 16 * x, bar(kBarRFull + rb));
                 }
-                if (ku > 0) wait(kBarKFree + kb, (ku - 1) & 1);
+                if (ku > 0) wait_idle(kBarKFree + kb, (ku - 1) & 1);
                 tc5::mbar_expect_tx(bar(kBarKFull + kb), (uint32_t)(it.ncols / 16) * 2048u);
                 for (int x = 0; x < it.ncols / 16; ++x)
                     tc5::tma_load_4d(k_u + kb * (kQItemCols * 128) + x * 2048, &tm_k, 0, h, node0 + 16 * x, b, bar(kBarKFull + kb));
-                if (j > 0) wait(kBarVFree, (j - 1) & 1);
+                if (j > 0) wait_idle(kBarVFree, (j - 1) & 1);
                 tc5::mbar_expect_tx(bar(kBarVFull), (uint32_t)(it.ncols / 16) * 2048u);
                 for (int x = 0; x < it.ncols / 16; ++x)
                     tc5::tma_load_4d(v_u + x * 2048, &tm_v, 0, h, node0 + 16 * x, b, bar(kBarVFull));
@@ -351,10 +355,10 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__
             for (int j = 0; j < J && !*abort_s; ++j) {
                 const Item it = items[j];
                 const int kb = j % kQKBufs, ku = j / kQKBufs;
-                if (it.flags & 1) { ++ci_a; wait(kBarRFull + (ci_a & 1), (ci_a >> 1) & 1); }
-                wait(kBarKFull + kb, ku & 1);
-                wait(kBarVFull, j & 1);
-                if (j > 0) wait(kBarSFree, (j - 1) & 1);   // every row thread holds its part of the item before
+                if (it.flags & 1) { ++ci_a; wait_idle(kBarRFull + (ci_a & 1), (ci_a >> 1) & 1); }
+                wait_idle(kBarKFull + kb, ku & 1);
+                wait_idle(kBarVFull, j & 1);
+                if (j > 0) wait_idle(kBarSFree, (j - 1) & 1);   // every row thread holds its part of the item before
                 if (*abort_s) break;
                 tc5::fence_after_sync();
                 const uint32_t k_lo = tc5::desc_lo_k_major(k_u + kb * (kQItemCols * 128));
@@ -382,7 +386,7 @@ bwd_q_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__
                 const Item it = items[j];
                 const int kb = j % kQKBufs;
                 if (it.flags & 1) ++ci_b;
-                wait(kBarDsFull, j & 1);
+                wait_idle(kBarDsFull, j & 1);
                 if (*abort_s) break;
                 tc5::fence_after_sync();
                 const uint32_t k_lo = tc5::desc_lo_mn_major(k_u + kb * (kQItemCols * 128));

@@ -173,11 +173,11 @@ size_t fwd_workspace_bytes(const bpt_graph& g, int B, int H, int d, bpt_dtype dt
 }
 
 // Two kernels cover the token rows: the warp-level one (mma.sync, 64-token tiles) and the tensor-memory
-// one (tcgen05 + TMA, 128-token tiles).  The second wins where a chunk holds enough nodes per token to
-// pay for its per-chunk hand-offs (measured at n = 8192: 0.32 against 0.34 ms at k = 64, 0.33 against 0.30 ms at
-// k = 48, 0.34 against 0.26 ms at k = 16; 6 to 12 % faster at k = 64 for n = 4096 .. 65536), so it takes k >= 56.
-// bpt_attn_options.path forces one of them for comparison runs.
-static bool want_tc5(int k, uint32_t path) { return path == BPT_PATH_TC5 || (path == BPT_PATH_AUTO && k >= 56); }
+// one (tcgen05 + TMA, 128-token tiles, two CTAs per SM).  Measured at n = 8192, left-only, batch 4 (ms, warp-level /
+// tensor-memory): k = 64 0.36 / 0.24, k = 48 0.32 / 0.22, k = 32 0.25 / 0.21, k = 24 0.25 / 0.21, k = 16 0.21 / 0.21,
+// k = 8 0.18 / 0.21, k = 4 0.18 / 0.23; bidirectional n = 16384, k = 16: 0.42 / 0.38; n = 65536, k = 64: 1.92 / 1.14.
+// The tensor-memory kernel therefore takes k >= 16.  bpt_attn_options.path forces one of them for comparison runs.
+static bool want_tc5(int k, uint32_t path) { return path == BPT_PATH_TC5 || (path == BPT_PATH_AUTO && k >= 16); }
 
 bpt_status launch_fwd(const AttnProblem& p) {
     if (tile_path(p.tree.n, p.tree.k, p.d, p.dtype == BPT_BF16)) {  // token rows and span rows on the tensor cores

@@ -152,6 +152,10 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__ r
         if (*abort_s) return;
         if (!tc5::mbar_wait_fast(bar(i), parity)) *abort_s = 1;
     };
+    auto wait_idle = [&](int i, uint32_t parity) {  // for the load and MMA threads
+        if (*abort_s) return;
+        if (!tc5::mbar_wait_idle(bar(i), parity)) *abort_s = 1;
+    };
 
     // ---- prologue: Q tile, the tile's node range per chunk, the item list, barriers, tensor memory ----
     for (int idx = tid; idx < kFTok * 8; idx += kFThreads) {
@@ -223,19 +227,19 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__ r
                 const int side = it.c >= n_left, level = side ? it.c - n_left : it.c;
                 const int node0 = node_id(t.n, level, 0) + crange[it.c].x + it.col0;
                 const int kb = j % kFBufs, ku = j / kFBufs;
-                if (ku > 0) wait(kFBarKFree + kb, (ku - 1) & 1);
+                if (ku > 0) wait_idle(kFBarKFree + kb, (ku - 1) & 1);
                 tc5::mbar_expect_tx(bar(kFBarKFull + kb), (uint32_t)(it.ncols / 16) * 2048u);
                 for (int x = 0; x < it.ncols / 16; ++x)
                     tc5::tma_load_4d(k_u + kb * (kFItemCols * 128) + x * 2048, &tm_k, 0, h, node0 + 16 * x, b, bar(kFBarKFull + kb));
                 if (it.flags & 1) {
                     ++ci;
-                    if (ci > 0) wait(kFBarRFree, (ci - 1) & 1);
+                    if (ci > 0) wait_idle(kFBarRFree, (ci - 1) & 1);
                     const int rel_base = it.c == 0 ? 0 : (side ? rel_right(t, level, 0) : rel_left(t, level, 0));
                     tc5::mbar_expect_tx(bar(kFBarRFull), (uint32_t)(rel_cols / 16) * 2048u);
                     for (int x = 0; x < rel_cols / 16; ++x)
                         tc5::tma_load_2d(r_u + x * 2048, &tm_r, 0, rel_base + 16 * x, bar(kFBarRFull));
                 }
-                if (ku > 0) wait(kFBarVFree + kb, (ku - 1) & 1);
+                if (ku > 0) wait_idle(kFBarVFree + kb, (ku - 1) & 1);
                 tc5::mbar_expect_tx(bar(kFBarVFull + kb), (uint32_t)(it.ncols / 16) * 2048u);
                 for (int x = 0; x < it.ncols / 16; ++x)
                     tc5::tma_load_4d(v_u + kb * (kFItemCols * 128) + x * 2048, &tm_v, 0, h, node0 + 16 * x, b, bar(kFBarVFull + kb));
@@ -250,9 +254,9 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__ r
             for (int j = 0; j < J && !*abort_s; ++j) {
                 const FItem it = items[j];
                 const int kb = j % kFBufs, ku = j / kFBufs;
-                if (it.flags & 1) { ++ci; wait(kFBarRFull, ci & 1); }
-                wait(kFBarKFull + kb, ku & 1);
-                if (j > 0) wait(kFBarSFree, (j - 1) & 1);   // every row thread holds its part of the item before
+                if (it.flags & 1) { ++ci; wait_idle(kFBarRFull, ci & 1); }
+                wait_idle(kFBarKFull + kb, ku & 1);
+                if (j > 0) wait_idle(kFBarSFree, (j - 1) & 1);   // every row thread holds its part of the item before
                 if (*abort_s) break;
                 tc5::fence_after_sync();
                 if (it.flags & 1) {
@@ -276,8 +280,8 @@ fwd_tc5_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__ r
             for (int j = 0; j < J && !*abort_s; ++j) {
                 const FItem it = items[j];
                 const int kb = j % kFBufs, ku = j / kFBufs;
-                wait(kFBarVFull + kb, ku & 1);
-                wait(kFBarPFull, j & 1);
+                wait_idle(kFBarVFull + kb, ku & 1);
+                wait_idle(kFBarPFull, j & 1);
                 if (*abort_s) break;
                 tc5::fence_after_sync();
                 const uint32_t v_lo = tc5::desc_lo_mn_major(v_u + kb * (kFItemCols * 128));

@@ -91,6 +91,19 @@ __device__ __forceinline__ bool mbar_wait_fast(uint32_t mbar, uint32_t parity, l
         }
     }
 }
+// The same for a thread that has nothing else to do and shares its scheduler with working warps (the load and
+// MMA-issue threads): each probe may suspend the thread for up to `hint_ns` until the phase completes, so
+// that the wait costs few issue slots.
+__device__ __forceinline__ bool mbar_wait_idle(uint32_t mbar, uint32_t parity, uint32_t hint_ns = 2000, long long limit = kWaitCycles) {
+    const long long start = clock64();
+    for (;;) {
+        uint32_t ok;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+                     : "=r"(ok) : "r"(mbar), "r"(parity), "r"(hint_ns) : "memory");
+        if (ok) return true;
+        if (clock64() - start > limit) return false;
+    }
+}
 __device__ __forceinline__ void mbar_arrive(uint32_t mbar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(mbar) : "memory");
 }
