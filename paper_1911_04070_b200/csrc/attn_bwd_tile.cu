@@ -550,13 +550,37 @@ bwd_tile_kernel(TreeParams t, ChunkPlan plan, BwdTileCfg cfg,
     }
 }
 
+// For every node and side the groups of tiles [first, last) whose chunk range covers the node: the same for every
+// (batch entry, head) pair, so it is found once per call (two bisections over the monotone table of group ranges)
+// and the gather reads it.
+__global__ void gather_plan_kernel(TreeParams t, ChunkPlan plan, const int2* __restrict__ tile_range, int tiles,
+                                   int2* __restrict__ node_tiles) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const int N = 2 * t.n - 1;
+    if (idx >= 2 * N) return;
+    const int vtx = idx >> 1, side = idx & 1;
+    const int l = node_level(t.n, vtx), m = vtx - node_id(t.n, l, 0);
+    int2 r = make_int2(0, 0);
+    if (l < (side ? plan.n_right : plan.n_left)) {
+        const int c = side ? plan.n_left + l : l;
+        const int2* tr = tile_range + (size_t)c * tiles;
+        int lo = 0, hi = tiles;  // first group whose range ends at or beyond m
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (tr[mid].y >= m) hi = mid; else lo = mid + 1; }
+        r.x = lo;
+        hi = tiles;              // first group whose range starts beyond m
+        while (lo < hi) { const int mid = (lo + hi) >> 1; if (tr[mid].x > m) hi = mid; else lo = mid + 1; }
+        r.y = lo;
+    }
+    node_tiles[idx] = r;
+}
+
 // dk, dv of every node: the partial rows of the tiles whose chunk range covers the node (both
 // sides), in tile order, plus for a token the row the span pass left for it (the affiliated
 // edges into its L ancestors).  One warp per (pair, node); lanes 0..15 hold four channels of dk
 // each, lanes 16..31 four channels of dv.
 __global__ void __launch_bounds__(256)
-bwd_gather_kernel(TreeParams t, ChunkPlan plan, const int2* __restrict__ tile_range, const float* __restrict__ slabs,
-                  const float* __restrict__ aff_slab,
+bwd_gather_kernel(TreeParams t, ChunkPlan plan, const int2* __restrict__ tile_range, const int2* __restrict__ node_tiles,
+                  const float* __restrict__ slabs, const float* __restrict__ aff_slab,
                   __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
                   int H, int pair0, int n_pairs, int tiles, float scale) {
     const int lane = threadIdx.x & 31;
@@ -572,16 +596,13 @@ bwd_gather_kernel(TreeParams t, ChunkPlan plan, const int2* __restrict__ tile_ra
     const float* slab_pair = slabs + (size_t)pl * tiles * tile_rows * 128;
 
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int4 nt = __ldg(reinterpret_cast<const int4*>(node_tiles) + vtx);  // (first, last) group of the left side, of the right side
+#pragma unroll
     for (int side = 0; side < 2; ++side) {
-        if (l >= (side ? plan.n_right : plan.n_left)) continue;
+        const int ta = side ? nt.z : nt.x, tb = side ? nt.w : nt.y;
+        if (ta >= tb) continue;
         const int c = side ? plan.n_left + l : l;
         const int2* tr = tile_range + (size_t)c * tiles;
-        int lo = 0, hi = tiles;  // first tile whose range ends at or beyond m
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if (tr[mid].y >= m) hi = mid; else lo = mid + 1; }
-        const int ta = lo;
-        hi = tiles;              // first tile whose range starts beyond m
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if (tr[mid].x > m) hi = mid; else lo = mid + 1; }
-        const int tb = lo;
         for (int T = ta; T < tb; ++T) {
             const int row = plan.slab_row0[c] + m - tr[T].x;
             const float4 x = __ldg(reinterpret_cast<const float4*>(slab_pair + ((size_t)T * tile_rows + row) * 128) + lane);
@@ -637,6 +658,7 @@ size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct TileWorkspace {
     int2* tile_range;
+    int2* node_tiles;   // per node and side the groups whose range covers it
     float *aff_slab, *ext_dq, *slabs, *drel_part, *drel_grp;
     int pairs_per_pass;
     size_t bytes;
@@ -671,6 +693,7 @@ TileWorkspace carve_tile(const TreeParams& t, const ChunkPlan& plan, size_t pair
     char* c = (char*)base;
     size_t off = 0;
     w.tile_range = (int2*)(c + off); off += align256(sizeof(int2) * chunks * tiles);
+    w.node_tiles = (int2*)(c + off); off += align256(sizeof(int2) * 2 * (size_t)(2 * t.n - 1));
     w.aff_slab = (float*)(c + off); off += align256(sizeof(float) * bwd_span_slab_floats(t, (int)pairs));
     w.ext_dq = (float*)(c + off); off += align256(sizeof(float) * bwd_span_ext_floats(t, (int)pairs));
     w.slabs = (float*)(c + off); off += align256(sizeof(float) * pairs * tiles * plan.slab_row0[chunks] * 128);
@@ -807,9 +830,13 @@ bpt_status launch_bwd_tile(const AttnProblem& p) {
             (const __nv_bfloat16*)p.rel_emb, (const __nv_bfloat16*)p.out, p.lse, (const __nv_bfloat16*)p.d_out,
             (__nv_bfloat16*)p.dq, ws.tile_range, ws.slabs, ws.drel_part, p.H, pair0, p.scale, p.lengths, p.drop);
         trace_mark(p.stream, "bwd_tile");
+        if (pair0 == 0) {  // the groups that cover every node: the same for all pairs
+            gather_plan_kernel<<<(2 * N + 255) / 256, 256, 0, p.stream>>>(t, plan, ws.tile_range, tiles, ws.node_tiles);
+            trace_mark(p.stream, "gather_plan");
+        }
         const int64_t warps = (int64_t)np * N;
         bwd_gather_kernel<<<(unsigned)((warps + 7) / 8), 256, 0, p.stream>>>(
-            t, plan, ws.tile_range, ws.slabs, ws.aff_slab, (__nv_bfloat16*)p.dk, (__nv_bfloat16*)p.dv,
+            t, plan, ws.tile_range, ws.node_tiles, ws.slabs, ws.aff_slab, (__nv_bfloat16*)p.dk, (__nv_bfloat16*)p.dv,
             p.H, pair0, np, tiles, p.scale);
         trace_mark(p.stream, "bwd_gather");
         drel_group_kernel<<<dim3((unsigned)((per_cta + 255) / 256), kDrelGroups), 256, 0, p.stream>>>(

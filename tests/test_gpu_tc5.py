@@ -34,6 +34,30 @@ def test_tensor_memory_forward_matches_oracle(n, k, flags, B, H):
     assert torch.equal(out, out2) and torch.equal(lse, lse2)
 
 
+@pytest.mark.parametrize("n,k,flags,B,H,std", [(256, 33, 1, 1, 3, 3.0), (1024, 64, 0, 1, 2, 3.0), (2048, 16, 0, 1, 2, 8.0),
+                                               (8192, 64, 1, 1, 2, 8.0)])
+def test_tensor_memory_forward_wide_logits(n, k, flags, B, H, std):
+    """Scores that differ by tens to hundreds of binary orders of magnitude between a row's items: the kernel keeps
+    its output accumulator in tensor memory and raises the row's reference exponent (rescaling the accumulator in
+    place) when a later item exceeds it, so this is the case that exercises the rescale."""
+    import torch
+    from oracle import ctwin
+    from paper_1911_04070_b200 import binding, synth
+    ref = ctwin.CGraph(n, k, flags)
+    x = synth.make_inputs(B, ref.n_nodes, H, 64, ref.n_rel, seed=11 + n + k, std_qkv=std, std_rel=0.3, bf16=True, with_grad=False)
+    g = binding.bpt_build_graph(n, k, flags, device="cuda:0", with_transpose=False)
+    t = {a: torch.from_numpy(b).to("cuda:0", torch.bfloat16) for a, b in x.items()}
+    ws = torch.empty(binding.bpt_attn_workspace_bytes(g, B, H, 64, binding.BPT_BF16, False), dtype=torch.uint8, device="cuda:0")
+    out, lse = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125, workspace=ws, path=binding.BPT_PATH_TC5)
+    assert binding.bpt_check(ws) == 0
+    o_ref, lse_ref = ctwin.attn_fwd(ref, x["q"], x["k"], x["v"], x["rel_emb"], 0.125)
+    assert np.isfinite(out.float().cpu().numpy()).all()
+    assert_close("out", out.float().cpu().numpy(), o_ref, TOL["bf16"])
+    assert_close("lse", lse.cpu().numpy(), lse_ref, TOL["bf16"])
+    out_m, lse_m = binding.bpt_attn_fwd(g, t["q"], t["k"], t["v"], t["rel_emb"], 0.125, path=binding.BPT_PATH_MMA)
+    assert_close("out vs warp-level kernel", out.float().cpu().numpy(), out_m.float().cpu().numpy(), TOL["bf16"])
+
+
 BWD_CASES = [
     # n, k, flags, B, H
     (128, 64, 0, 2, 2),       # one tile per kernel, k = 64 on both sides
