@@ -41,9 +41,9 @@ GATHER_BYTES_PER_EDGE_HEAD = {  # algorithmic bytes of the gather model, per edg
 # Which part of the gather model each kernel carries: (passes, "token" | "span" | "all" destination rows).
 KERNEL_MODEL = {
     "fwd_rows": (("fwd",), "all"), "bwd_dst": (("bwd_dst",), "all"), "bwd_src": (("bwd_src",), "all"),
-    "fwd_tile": (("fwd",), "token"), "fwd_tc5": (("fwd",), "token"), "fwd_span": (("fwd",), "span"),
+    "fwd_tile": (("fwd",), "token"), "fwd_tc5": (42.29e6 / 8, "attn_fwd_tc5.cu", "dd6a011e4b77f820"),
     "bwd_tile": (("bwd_dst", "bwd_src"), "token"), "bwd_span": (("bwd_dst", "bwd_src"), "span"),
-    "bwd_q_tc5": (("bwd_dst",), "token"), "bwd_kv_tc5": (("bwd_src",), "token"),
+    "bwd_q_tc5": (60.69e6 / 8, "attn_bwd_q_tc5.cu", "306dd7c8ce99ac47"),
 }
 # DRAM bytes (read + write) per (batch entry, head) pair of one launch, from ncu captures of the character-LM
 # shape at batch 1 (n = 8192, k = 64, left-only, 8 heads; every pair is an independent problem, so traffic
@@ -51,9 +51,9 @@ KERNEL_MODEL = {
 # were read; when the file has changed since, the bench reports traffic = null instead of a stale number.
 NCU_DRAM_BYTES_PER_PAIR = {
     # kernel: (bytes per pair, source file, sha256 of the file at capture time (first 16 hex digits))
-    "fwd_tc5": (41.22e6 / 8, "attn_fwd_tc5.cu", "812e238b1a1e6f78"),
-    "bwd_q_tc5": (60.39e6 / 8, "attn_bwd_q_tc5.cu", "d3e9f827fddbbe6a"),
-    "bwd_kv_tc5": (118.41e6 / 8, "attn_bwd_kv_tc5.cu", "e39a0a104ddf814d"),
+    "fwd_tc5": (42.29e6 / 8, "attn_fwd_tc5.cu", "dd6a011e4b77f820"),
+    "bwd_q_tc5": (60.69e6 / 8, "attn_bwd_q_tc5.cu", "306dd7c8ce99ac47"),
+    "bwd_kv_tc5": (113.88e6 / 8, "attn_bwd_kv_tc5.cu", "3c537c76ec9adbce"),
 }
 FLOPS_PER_EDGE_HEAD = {"fwd": 6, "bwd": 14}   # x d_head: q.k, q.r, P.v forward; s again, dP, dq, dk, dv, d_rel backward
 
