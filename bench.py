@@ -41,9 +41,9 @@ GATHER_BYTES_PER_EDGE_HEAD = {  # algorithmic bytes of the gather model, per edg
 # Which part of the gather model each kernel carries: (passes, "token" | "span" | "all" destination rows).
 KERNEL_MODEL = {
     "fwd_rows": (("fwd",), "all"), "bwd_dst": (("bwd_dst",), "all"), "bwd_src": (("bwd_src",), "all"),
-    "fwd_tile": (("fwd",), "token"), "fwd_tc5": (42.29e6 / 8, "attn_fwd_tc5.cu", "dd6a011e4b77f820"),
+    "fwd_tile": (("fwd",), "token"), "fwd_tc5": (("fwd",), "token"), "fwd_span": (("fwd",), "span"),
     "bwd_tile": (("bwd_dst", "bwd_src"), "token"), "bwd_span": (("bwd_dst", "bwd_src"), "span"),
-    "bwd_q_tc5": (60.69e6 / 8, "attn_bwd_q_tc5.cu", "306dd7c8ce99ac47"),
+    "bwd_q_tc5": (("bwd_dst",), "token"), "bwd_kv_tc5": (("bwd_src",), "token"),
 }
 # DRAM bytes (read + write) per (batch entry, head) pair of one launch, from ncu captures of the character-LM
 # shape at batch 1 (n = 8192, k = 64, left-only, 8 heads; every pair is an independent problem, so traffic

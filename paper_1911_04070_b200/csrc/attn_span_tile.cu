@@ -244,7 +244,7 @@ fwd_span_kernel(TreeParams t, const __nv_bfloat16* __restrict__ q, const __nv_bf
 }
 
 // Outer ancestors of the forward: merge the tiles' partial states in tile order.
-// One warp per (pair, span); lane c holds channels 2c, 2c + 1.
+// One warp per (pair, span), the root first; lane c holds channels 2c, 2c + 1.
 __global__ void __launch_bounds__(128)
 fwd_span_merge_kernel(TreeParams t, const float* __restrict__ ext_part, __nv_bfloat16* __restrict__ out,
                       float* __restrict__ lse, int H, int n_pairs, int tiles, int n_ext) {
@@ -258,36 +258,44 @@ fwd_span_merge_kernel(TreeParams t, const float* __restrict__ ext_part, __nv_bfl
     const int T0 = mi << (j - kInnerLevels), nT = 1 << (j - kInnerLevels);
     const float* base = ext_part + (((size_t)pair * tiles + T0) * n_ext + e) * kExtStride;
     const size_t stride = (size_t)n_ext * kExtStride;
-    // lane t takes tiles t, t + 32, ...; the lanes' sums are then added in a fixed butterfly order
+    // Lane c holds channels 2c, 2c + 1 and adds the tiles' rows in tile order (coalesced row loads); the tiles'
+    // rescaling factors are computed 32 at a time, one per lane, and handed round by shuffle.
     float mx = -INFINITY;
     for (int x = lane; x < nT; x += 32) mx = fmaxf(mx, base[(size_t)x * stride]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (mx == -INFINITY) mx = 0.f;  // a span without real tokens: every partial is empty (2^-inf = 0 below)
-    float l = 0.f, acc[64];
+    float l = 0.f, a0 = 0.f, a1 = 0.f;
+    for (int x0 = 0; x0 < nT; x0 += 32) {
+        float f = 0.f, lf = 0.f;
+        if (x0 + lane < nT) {
+            const float* p = base + (size_t)(x0 + lane) * stride;
+            f = fast_exp2(p[0] - mx);
+            lf = p[1] * f;
+        }
 #pragma unroll
-    for (int c = 0; c < 64; ++c) acc[c] = 0.f;
-    for (int x = lane; x < nT; x += 32) {
-        const float* p = base + (size_t)x * stride;
-        const float f = fast_exp2(p[0] - mx);
-        l = fmaf(p[1], f, l);
+        for (int o = 16; o > 0; o >>= 1) lf += __shfl_xor_sync(0xffffffffu, lf, o);
+        l += lf;
+        const float* row = base + (size_t)x0 * stride + 2 + 2 * lane;
+        if (x0 + 32 <= nT) {
+            float2 a[32];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            const float2 a = *reinterpret_cast<const float2*>(p + 2 + 2 * c);
-            acc[2 * c] = fmaf(a.x, f, acc[2 * c]);
-            acc[2 * c + 1] = fmaf(a.y, f, acc[2 * c + 1]);
+            for (int i = 0; i < 32; ++i) a[i] = *reinterpret_cast<const float2*>(row + (size_t)i * stride);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float fi = __shfl_sync(0xffffffffu, f, i);
+                a0 = fmaf(a[i].x, fi, a0);
+                a1 = fmaf(a[i].y, fi, a1);
+            }
+        } else {
+            for (int i = 0; i < nT - x0; ++i) {
+                const float fi = __shfl_sync(0xffffffffu, f, i);
+                const float2 a = *reinterpret_cast<const float2*>(row + (size_t)i * stride);
+                a0 = fmaf(a.x, fi, a0);
+                a1 = fmaf(a.y, fi, a1);
+            }
         }
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        l += __shfl_xor_sync(0xffffffffu, l, o);
-#pragma unroll
-        for (int c = 0; c < 64; ++c) acc[c] += __shfl_xor_sync(0xffffffffu, acc[c], o);
-    }
-    float a0 = 0.f, a1 = 0.f;  // this lane's two channels (static register indices only)
-#pragma unroll
-    for (int c = 0; c < 32; ++c)
-        if (c == lane) { a0 = acc[2 * c]; a1 = acc[2 * c + 1]; }
     const float inv = l > 0.f ? 1.f / l : 0.f;  // l = 0: a span without real tokens
     const size_t rs = (size_t)H * 64;
     *reinterpret_cast<uint32_t*>(out + ((size_t)b * (2 * t.n - 1) + node) * rs + (size_t)h * 64 + lane * 2) = pack_bf16(a0 * inv, a1 * inv);
