@@ -6,10 +6,10 @@
 // One CTA = 128 rows = the 128 lanes of tensor memory; the whole output row (D <= 512 channels) stays in
 // tensor memory as fp32, so the residual add and both normalisation passes run on it without a trip through
 // HBM.  A load thread brings a [128 x 64] and w_o [D x 64] k-blocks in with TMA (two stages, no multicast), an
-// MMA thread issues tcgen05.mma (N = min(D, 256) columns per instruction), four epilogue warps (one thread per
-// row) add the residual into tensor memory, take mean and variance in two further sweeps, normalise, and stage
-// the bf16 rows in shared memory for coalesced stores.  Every wait is bounded; a give-up is reported through the
-// status word.
+// MMA thread issues tcgen05.mma (N = min(D, 256) columns per instruction), sixteen epilogue warps (four threads
+// per row, a quarter of the columns each; the row statistics pass between them through shared memory) add the
+// residual into tensor memory, take mean and variance in two further sweeps, normalise, and stage the bf16 rows in
+// shared memory for coalesced stores.  Every wait is bounded; a give-up is reported through the status word.
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"
 #include "tc5_host.cuh"
@@ -20,7 +20,9 @@ namespace bpt {
 namespace {
 
 constexpr int kOpRows = 128;
-constexpr int kOpThreads = 6 * 32;   // four epilogue warps, a load warp, an MMA warp
+constexpr int kOpTpr = 4;                              // epilogue threads per row
+constexpr int kOpEpiWarps = 4 * kOpTpr;
+constexpr int kOpThreads = (kOpEpiWarps + 2) * 32;     // epilogue warps, a load warp, an MMA warp
 constexpr int kOpStages = 2;
 constexpr int kOpMaxD = 512;
 
@@ -37,7 +39,7 @@ inline OpSmem op_smem(int D) {
     s.out_stride = D * 2 + 16;
     const int staging = kOpRows * s.out_stride;
     if (s.bar_off < staging) s.bar_off = (staging + 1023) & ~1023;
-    s.bytes = (size_t)s.bar_off + 128 + 1024;
+    s.bytes = (size_t)s.bar_off + 128 + kOpTpr * kOpRows * 4 + 1024;   // barriers, then the exchange of row statistics
     return s;
 }
 
@@ -50,6 +52,7 @@ out_proj_norm_kernel(const __nv_bfloat16* __restrict__ h, const float* __restric
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + cfg.bar_off);   // full[2], empty[2], done
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 5);
     volatile int* abort_s = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* xch_s = reinterpret_cast<float*>(smem + cfg.bar_off + 128);   // [kOpTpr][128 rows]
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const long long row0 = (long long)blockIdx.x * kOpRows;
     const uint32_t s_u = smem_u32(smem), bar_u = smem_u32(bars);
@@ -72,7 +75,7 @@ out_proj_norm_kernel(const __nv_bfloat16* __restrict__ h, const float* __restric
     tc5::fence_after_sync();
     const uint32_t tbase = *tmem_slot;
 
-    if (w == 4) {
+    if (w == kOpEpiWarps) {
         // =============== load warp: k-blocks of a and w_o, two stages ===============
         if (lane == 0) {
             for (int kb = 0; kb < n_kb && !*abort_s; ++kb) {
@@ -85,7 +88,7 @@ out_proj_norm_kernel(const __nv_bfloat16* __restrict__ h, const float* __restric
                     tc5::tma_load_2d(dst + cfg.a_bytes + nb * 128, &tm_w, kb * 64, nb, bar(st));
             }
         }
-    } else if (w == 5) {
+    } else if (w == kOpEpiWarps + 1) {
         // =============== MMA warp: acc[128 x D] += a_kb w_kb^T ===============
         if (lane == 0) {
             const int n_half = D > 256 ? 2 : 1, n_cols = D > 256 ? 256 : D;
@@ -106,24 +109,49 @@ out_proj_norm_kernel(const __nv_bfloat16* __restrict__ h, const float* __restric
             tc5::commit(bar(4));
         }
     } else {
-        // =============== epilogue warps: one thread per row ===============
-        const int r = w * 32 + lane;
-        const uint32_t lane_base = (uint32_t)(w * 32) << 16;
+        // =============== epilogue warps: four threads per row, D / 4 consecutive columns each ===============
+        const int quad = w & 3, part = w >> 2;
+        const int r = quad * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
         const long long row = row0 + r;
         const bool live = row < rows;
+        const int c_lo = part * (D / kOpTpr), c_hi = c_lo + D / kOpTpr;
+        auto row_sum = [&](float v) {   // sum over the row's threads (the warps that share a lane quadrant)
+            xch_s[part * kOpRows + r] = v;
+            switch (quad) {
+                case 0: asm volatile("bar.sync 1, %0;" ::"n"(32 * kOpTpr) : "memory"); break;
+                case 1: asm volatile("bar.sync 2, %0;" ::"n"(32 * kOpTpr) : "memory"); break;
+                case 2: asm volatile("bar.sync 3, %0;" ::"n"(32 * kOpTpr) : "memory"); break;
+                default: asm volatile("bar.sync 4, %0;" ::"n"(32 * kOpTpr) : "memory"); break;
+            }
+            float t = 0.f;
+#pragma unroll
+            for (int x = 0; x < kOpTpr; ++x) t += xch_s[x * kOpRows + r];
+            return t;
+        };
+        auto quad_sync = [&]() {        // before the exchange slots are written again
+            switch (quad) {
+                case 0: asm volatile("bar.sync 1, %0;" ::"n"(32 * kOpTpr) : "memory"); break;
+                case 1: asm volatile("bar.sync 2, %0;" ::"n"(32 * kOpTpr) : "memory"); break;
+                case 2: asm volatile("bar.sync 3, %0;" ::"n"(32 * kOpTpr) : "memory"); break;
+                default: asm volatile("bar.sync 4, %0;" ::"n"(32 * kOpTpr) : "memory"); break;
+            }
+        };
         wait(4, 0);
         tc5::fence_after_sync();
         const uint4* hrow = reinterpret_cast<const uint4*>(h + (live ? row : 0) * (long long)D);
         // sweep 1: x = acc + h back into tensor memory, and the row sum
         float sum = 0.f;
-        for (int c = 0; c < D; c += 32) {
+        for (int c = c_lo; c < c_hi; c += 32) {
             uint32_t x[32];
             tc5::tmem_ld32(tbase + lane_base + c, x);
+            uint4 hv[4];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) hv[q4] = live ? __ldg(hrow + (c >> 3) + q4) : make_uint4(0, 0, 0, 0);
             tc5::tmem_ld_wait();
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
-                const uint4 hv = live ? __ldg(hrow + (c >> 3) + q4) : make_uint4(0, 0, 0, 0);
-                const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+                const uint32_t hw[4] = {hv[q4].x, hv[q4].y, hv[q4].z, hv[q4].w};
 #pragma unroll
                 for (int y = 0; y < 4; ++y) {
                     const float v0 = __uint_as_float(x[q4 * 8 + 2 * y]) + __uint_as_float(hw[y] << 16);
@@ -136,20 +164,21 @@ out_proj_norm_kernel(const __nv_bfloat16* __restrict__ h, const float* __restric
             tc5::tmem_st32(tbase + lane_base + c, x);
         }
         tc5::tmem_st_wait();
-        const float mean = sum / (float)D;
+        const float mean = row_sum(sum) / (float)D;
         // sweep 2: the variance about the mean
         float ssq = 0.f;
-        for (int c = 0; c < D; c += 32) {
+        for (int c = c_lo; c < c_hi; c += 32) {
             uint32_t x[32];
             tc5::tmem_ld32(tbase + lane_base + c, x);
             tc5::tmem_ld_wait();
 #pragma unroll
             for (int y = 0; y < 32; ++y) { const float d = __uint_as_float(x[y]) - mean; ssq = fmaf(d, d, ssq); }
         }
-        const float rstd = rsqrtf(ssq / (float)D + eps);
+        quad_sync();   // every thread of the row has read the sums
+        const float rstd = rsqrtf(row_sum(ssq) / (float)D + eps);
         // the stage buffers are free (every product has completed): stage the normalised rows there
         unsigned char* orow = smem + (size_t)r * cfg.out_stride;
-        for (int c = 0; c < D; c += 32) {
+        for (int c = c_lo; c < c_hi; c += 32) {
             uint32_t x[32];
             tc5::tmem_ld32(tbase + lane_base + c, x);
             tc5::tmem_ld_wait();
