@@ -764,7 +764,9 @@ size_t tc5_pairs_for_budget(const TreeParams& t, int B, int H, size_t budget) {
 // enough nodes per token; bpt_attn_options.path forces either family.
 bool want_bwd_tc5(const TreeParams& t, uint32_t path) {
     if (path == BPT_PATH_MMA || !bwd_q_tc5_fits(t)) return false;
-    return path == BPT_PATH_TC5 || t.k >= 56;   // measured at n = 1024 .. 65536: ahead of the warp-level kernels at k = 64, level at k = 48
+    // measured (ms, warp-level / tensor-memory): k = 48: n = 8192 left-only 1.40 / 1.36, n = 4096 2.17 / 1.97, n = 16384 2.78 / 2.42,
+    // n = 1024 1.57 / 1.58; k = 40: n = 8192 left-only 1.31 / 1.36, n = 4096 2.00 / 1.97; k = 64: ahead at every n
+    return path == BPT_PATH_TC5 || t.k >= 48;
 }
 
 bpt_status launch_bwd_tc5(const AttnProblem& p) {

@@ -88,6 +88,7 @@ SMALL = [
     (256, 33, 1, 1, 3, 64, True),      # odd k, left only
     (512, 63, 2, 1, 2, 64, True),      # Algorithm-1 graph, k + 1 = 64 relation rows exactly
     (4096, 64, 0, 1, 1, 64, True),     # k = 64 on both sides over 64 tiles
+    (1024, 48, 0, 1, 2, 64, True),     # smallest k at which both passes take the tensor-memory kernels by themselves
 ]
 
 
