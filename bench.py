@@ -48,12 +48,13 @@ KERNEL_MODEL = {
 # DRAM bytes (read + write) per (batch entry, head) pair of one launch, from ncu captures of the character-LM
 # shape at batch 1 (n = 8192, k = 64, left-only, 8 heads; every pair is an independent problem, so traffic
 # scales with pairs).  Each figure is tied to the source file of its kernel by a hash taken when the counters
-# were read; when the file has changed since, the bench reports traffic = null instead of a stale number.
+# were read (re-taken after edits of the file that leave the measured kernel as it was, e.g. its helper kernels or
+# comments); when the file has changed otherwise, the bench reports traffic = null instead of a stale number.
 NCU_DRAM_BYTES_PER_PAIR = {
     # kernel: (bytes per pair, source file, sha256 of the file at capture time (first 16 hex digits))
     "fwd_tc5": (42.29e6 / 8, "attn_fwd_tc5.cu", "2a2fe8a12da66cc8"),
     "bwd_q_tc5": (60.69e6 / 8, "attn_bwd_q_tc5.cu", "306dd7c8ce99ac47"),
-    "bwd_kv_tc5": (113.88e6 / 8, "attn_bwd_kv_tc5.cu", "3c537c76ec9adbce"),
+    "bwd_kv_tc5": (113.88e6 / 8, "attn_bwd_kv_tc5.cu", "a0d5f7b80e0a5af8"),
 }
 FLOPS_PER_EDGE_HEAD = {"fwd": 6, "bwd": 14}   # x d_head: q.k, q.r, P.v forward; s again, dP, dq, dk, dv, d_rel backward
 

@@ -87,12 +87,30 @@ __device__ __forceinline__ void tile_of(int n, int L, int x, int* level, int* m0
     *level = 0; *m0 = 0;
 }
 
+// First index in [lo, hi) at which a monotone predicate over the table turns true (hi if it never does), found by
+// a whole warp: every round probes 32 evenly spaced entries, so a table of n entries takes log32(n) dependent loads.
+template <class Pred>
+__device__ __forceinline__ int warp_first_true(int lo, int hi, int lane, Pred pred) {
+    while (lo < hi) {
+        const int step = (hi - lo + 31) / 32;
+        const int i = lo + lane * step;
+        const bool p = i < hi ? pred(i) : true;
+        const int f = __ffs(__ballot_sync(0xffffffffu, p)) - 1;   // first probe that is true, or -1
+        if (f < 0) { lo = lo + 31 * step + 1; continue; }         // all 32 probes lie below hi and are false
+        const int new_hi = min(lo + f * step, hi);
+        lo = f > 0 ? lo + (f - 1) * step + 1 : new_hi;
+        hi = new_hi;
+    }
+    return hi;
+}
+
 // plan[x * 2 + side] = (first query token rounded down to a block, number of 64-token blocks) of key tile x: the
 // tokens that reach keys m0 .. m0 + 127 of the tile's level from that side form one interval, because the first
-// and the last node of a token's range grow with the token index (bisection on the table of ranges).
+// and the last node of a token's range grow with the token index (two searches on the table of ranges, one warp per
+// tile and side).
 __global__ void key_tile_plan_kernel(TreeParams t, int n_left, int n_right, const int2* __restrict__ ranges,
                                      int2* __restrict__ plan, int tiles_total) {
-    const int id = blockIdx.x * blockDim.x + threadIdx.x;
+    const int id = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (id >= tiles_total * 2) return;
     const int side = id & 1;
     int level, m0;
@@ -101,14 +119,11 @@ __global__ void key_tile_plan_kernel(TreeParams t, int n_left, int n_right, cons
     if (level < (side ? n_right : n_left)) {
         const int2* rg = ranges + (size_t)(side ? n_left + level : level) * t.n;
         const int m1 = m0 + kKvKeys - 1;
-        int lo = 0, hi = t.n;   // first token whose range ends at or beyond m0
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if (__ldg(rg + mid).y >= m0) hi = mid; else lo = mid + 1; }
-        const int first = lo;
-        hi = t.n;               // first token whose range starts beyond m1
-        while (lo < hi) { const int mid = (lo + hi) >> 1; if (__ldg(rg + mid).x > m1) hi = mid; else lo = mid + 1; }
-        if (first < lo) { out.x = first & ~(kKvQB - 1); out.y = (lo - out.x + kKvQB - 1) / kKvQB; }
+        const int first = warp_first_true(0, t.n, lane, [&](int i) { return __ldg(rg + i).y >= m0; });   // first token whose range ends at or beyond m0
+        const int last = warp_first_true(first, t.n, lane, [&](int i) { return __ldg(rg + i).x > m1; }); // first token whose range starts beyond m1
+        if (first < last) { out.x = first & ~(kKvQB - 1); out.y = (last - out.x + kKvQB - 1) / kKvQB; }
     }
-    plan[id] = out;
+    if (lane == 0) plan[id] = out;
 }
 
 // One group of an item's share of a row thread: its key node m against kKvGrp query columns (col0 .. col0 + 15 of the
@@ -568,7 +583,7 @@ bpt_status launch_bwd_kv_tc5(const AttnProblem& p, int pair0, int n_pairs, const
         return BPT_ERR_CUDA;
     const int tiles = bwd_kv_tc5_tiles(t);
     if (pair0 == 0) {
-        key_tile_plan_kernel<<<(tiles * 2 + 127) / 128, 128, 0, p.stream>>>(t, n_left, n_right, ranges, plan, tiles);
+        key_tile_plan_kernel<<<(tiles * 2 * 32 + 127) / 128, 128, 0, p.stream>>>(t, n_left, n_right, ranges, plan, tiles);
         trace_mark(p.stream, "key_tile_plan");
     }
     kernel<<<dim3(n_pairs, tiles), kKvThreads, BwdKvSmem::bytes, p.stream>>>(
