@@ -52,9 +52,9 @@ KERNEL_MODEL = {
 # comments); when the file has changed otherwise, the bench reports traffic = null instead of a stale number.
 NCU_DRAM_BYTES_PER_PAIR = {
     # kernel: (bytes per pair, source file, sha256 of the file at capture time (first 16 hex digits))
-    "fwd_tc5": (42.29e6 / 8, "attn_fwd_tc5.cu", "2a2fe8a12da66cc8"),
-    "bwd_q_tc5": (60.69e6 / 8, "attn_bwd_q_tc5.cu", "306dd7c8ce99ac47"),
-    "bwd_kv_tc5": (113.88e6 / 8, "attn_bwd_kv_tc5.cu", "a0d5f7b80e0a5af8"),
+    "fwd_tc5": (42.29e6 / 8, "attn_fwd_tc5.cu", "2f9c6b763080e59f"),
+    "bwd_q_tc5": (60.69e6 / 8, "attn_bwd_q_tc5.cu", "d4456f5a3fecb677"),
+    "bwd_kv_tc5": (113.88e6 / 8, "attn_bwd_kv_tc5.cu", "2342321c21ce8852"),
 }
 FLOPS_PER_EDGE_HEAD = {"fwd": 6, "bwd": 14}   # x d_head: q.k, q.r, P.v forward; s again, dP, dq, dk, dv, d_rel backward
 

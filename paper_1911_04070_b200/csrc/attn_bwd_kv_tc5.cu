@@ -18,7 +18,7 @@
 // CTA and is written once, rounded once; there are no partial rows and no atomics.  The per-CTA d_rel
 // partials ((k + 2) x 64 floats per side) are summed in a fixed order by drel_kv_reduce_kernel.
 //
-// A load warp keeps a ring of three (Q_blk, dO_blk) buffers full with TMA (no multicast) and computes
+// A load warp keeps a ring of three (Q_blk, dO_blk) buffers full with TMA (each CTA its own copies) and computes
 // each block's per-query facts (node range at this level, lse, row term); an MMA warp issues the
 // products; mbarriers carry the hand-offs; every wait is bounded and a give-up is reported through the
 // status word while the kernel runs to its end without waiting again.

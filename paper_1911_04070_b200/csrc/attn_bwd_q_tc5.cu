@@ -15,7 +15,7 @@
 // issued with the chunk's last item).  dQ stays in tensor memory for the whole tile.
 //
 // Pipeline: the load thread keeps three K buffers, one V buffer and two R buffers full with TMA
-// (cp.async.bulk.tensor, no multicast); every hand-off is an mbarrier; every wait is bounded and a
+// (cp.async.bulk.tensor, each CTA its own copies); every hand-off is an mbarrier; every wait is bounded and a
 // give-up is reported through the status word while the kernel runs to its end without waiting again.
 #include "bpt_internal.cuh"
 #include "mma_tools.cuh"

@@ -23,7 +23,7 @@
 // The kernel is sized for two CTAs per SM (at most 112 KB of shared memory, 256 tensor-memory columns,
 // 80 registers): while one tile waits for a product, a copy or a barrier the other one computes.  A
 // load thread keeps two K and two V buffers and one R buffer full with TMA (cp.async.bulk.tensor, 16-row
-// boxes straight into the 128-byte-swizzled layout the tensor core reads, no multicast); every hand-off
+// boxes straight into the 128-byte-swizzled layout the tensor core reads, each CTA its own copies); every hand-off
 // is an mbarrier; the load and MMA threads suspend in their waits instead of spinning; every wait is
 // bounded and a give-up is reported through the status word while the kernel runs to its end without
 // waiting again.  The per-token node ranges come from a table (one entry per chunk and token) that a small

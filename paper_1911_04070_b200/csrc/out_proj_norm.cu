@@ -5,7 +5,7 @@
 //
 // One CTA = 128 rows = the 128 lanes of tensor memory; the whole output row (D <= 512 channels) stays in
 // tensor memory as fp32, so the residual add and both normalisation passes run on it without a trip through
-// HBM.  A load thread brings a [128 x 64] and w_o [D x 64] k-blocks in with TMA (two stages, no multicast), an
+// HBM.  A load thread brings a [128 x 64] and w_o [D x 64] k-blocks in with TMA (two stages, each CTA its own copies), an
 // MMA thread issues tcgen05.mma (N = min(D, 256) columns per instruction), sixteen epilogue warps (four threads
 // per row, a quarter of the columns each; the row statistics pass between them through shared memory) add the
 // residual into tensor memory, take mean and variance in two further sweeps, normalise, and stage the bf16 rows in

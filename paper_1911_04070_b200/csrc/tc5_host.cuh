@@ -1,7 +1,7 @@
 // Host side of the TMA loads of the tensor-memory kernels: tensor maps over the node-major
 // [B, N, H, 64] bf16 tensors and the [n_rel, 64] relation table.  A box is 16 consecutive rows of 64
 // elements of one (batch entry, head), written to shared memory in the 128-byte swizzle the tensor
-// core reads.  The maps cover this GPU's own memory only and no load uses cluster multicast.
+// core reads.  The maps cover this GPU's own memory only and every CTA issues its own loads.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>

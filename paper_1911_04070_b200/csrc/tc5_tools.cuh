@@ -112,7 +112,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t mbar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(mbar), "r"(bytes) : "memory");
 }
 
-// TMA tile loads (no multicast): the box of the tensor map at the given coordinates -> shared memory,
+// TMA tile loads (plain, one destination CTA): the box of the tensor map at the given coordinates -> shared memory,
 // completion counted in bytes on the mbarrier.  The innermost coordinate is always 0 here (16-byte rule).
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int c0, int c1, int c2, int c3, uint32_t mbar) {
     asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
